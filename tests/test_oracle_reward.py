@@ -1,0 +1,196 @@
+"""Pins for the Draft Tree Reward (Eq. 3-5) and the greedy accepted path."""
+import itertools
+
+import numpy as np
+import pytest
+from scipy.special import logsumexp, softmax
+
+from oracle import gto_oracle as orc
+from test_oracle_tree import node_paths
+
+
+def tiny_case(seed, V=3, D=3, k=2, g=5, scale=1.5):
+    rng = np.random.default_rng(seed)
+    draft = rng.normal(size=(D, k, V)) * scale
+    target = rng.normal(size=(1 + (D - 1) * k, V)) * scale
+    tree = orc.build_tree(draft, D, k, g)
+    return draft, target, tree
+
+
+def rollout_dist(tree, target, prefix):
+    """Target next-token distribution after `prefix` (a tuple of tokens): the tree's
+    own context row while the prefix is the root or an expanded tree node, else any
+    fixed distribution (uniform) - it cannot change a match count any more."""
+    V = target.shape[1]
+    if len(prefix) == 0:
+        return softmax(target[0])
+    paths = node_paths(tree)
+    if prefix in paths:
+        n = paths.index(prefix)
+        if tree.slot[n] >= 0 and tree.depth[n] < tree.D:
+            return softmax(target[orc.context_row(int(tree.depth[n]), int(tree.slot[n]), tree.k)])
+    return np.full(V, 1.0 / V)
+
+
+def lcp(a, b):
+    n = 0
+    for x, y in zip(a, b):
+        if x != y:
+            break
+        n += 1
+    return n
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_sequence_length_is_expected_leading_matches_by_enumeration(seed):
+    """Eq. 3: L_i is the expected number of leading tokens of S_i that a target
+    roll-out reproduces.  Enumerate every roll-out of length D."""
+    draft, target, tree = tiny_case(seed)
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    paths = node_paths(tree)
+    V, D = target.shape[1], tree.D
+    exp_match = np.zeros(tree.g)
+    exp_max = 0.0
+    total = 0.0
+    leaves = [paths[i] for i in rw["leaves"]]
+    for x in itertools.product(range(V), repeat=D):
+        pr = 1.0
+        for u in range(D):
+            pr *= rollout_dist(tree, target, x[:u])[x[u]]
+        total += pr
+        for n in range(tree.g):
+            exp_match[n] += pr * lcp(x, paths[n])
+        exp_max += pr * max(lcp(x, s) for s in leaves)
+    assert abs(total - 1.0) < 1e-12
+    assert np.allclose(exp_match, rw["Lc"], atol=1e-12)
+    # exact tree acceptance: E[max_i matches] = sum_n Pp_n, between max L and sum L
+    assert abs(exp_max - rw["etree"]) < 1e-12
+    L = rw["Lc"][rw["leaves"]]
+    assert L.max() - 1e-12 <= rw["etree"] <= L.sum() + 1e-12
+    # Eq. 5 with eta = 1 and the App. A Eq. (1) bounds
+    assert abs(rw["r"] - logsumexp(L)) < 1e-12
+    assert L.max() <= rw["r"] <= L.max() + np.log(len(L)) + 1e-12
+
+
+def test_sequence_length_by_monte_carlo():
+    draft, target, tree = tiny_case(11, V=4, D=3, k=2, g=6)
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    paths = node_paths(tree)
+    rng = np.random.default_rng(0)
+    n_roll = 100000
+    counts = np.zeros((n_roll, tree.g))
+    for i in range(n_roll):
+        x = ()
+        for u in range(tree.D):
+            q = rollout_dist(tree, target, x)
+            x = x + (int(rng.choice(len(q), p=q)),)
+        counts[i] = [lcp(x, s) for s in paths]
+    mean = counts.mean(axis=0)
+    sem = counts.std(axis=0) / np.sqrt(n_roll) + 1e-9
+    assert np.all(np.abs(mean - rw["Lc"]) < 4.5 * sem)
+
+
+@pytest.mark.parametrize("n_match", [0, 1, 3, 5])
+def test_single_chain_one_hot_reward_counts_matching_tokens(n_match):
+    """k = 1, g = D: the tree is one chain; with one-hot target rows the reward is
+    the number of leading draft tokens equal to the target's tokens."""
+    rng = np.random.default_rng(n_match)
+    D, V = 5, 20
+    draft = rng.normal(size=(D, 1, V))
+    tree = orc.build_tree(draft, D, 1, D)
+    target = np.full((D, V), -1000.0)
+    for d in range(D):
+        tok = int(tree.token[d])
+        hot = tok if d < n_match else (tok + 1) % V
+        target[d, hot] = 1000.0
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    assert rw["r"] == pytest.approx(float(n_match), abs=1e-12)
+    assert len(rw["leaves"]) == 1
+    path = orc.longest_accepted(tree, target)
+    assert len(path["nodes"]) == n_match
+    assert path["nodes"] == list(range(n_match))
+
+
+def test_eta_limits_and_variants():
+    draft, target, tree = tiny_case(5, V=6, D=4, k=3, g=12)
+    p, _ = orc.target_node_probs(tree, target)
+    L = orc.tree_reward(tree, p)["Lc"][orc.tree_reward(tree, p)["leaves"]]
+    assert orc.tree_reward(tree, p, eta=200.0)["r"] == pytest.approx(L.max(), abs=2e-2)
+    small = 1e-5
+    assert orc.tree_reward(tree, p, eta=small)["r"] - np.log(len(L)) / small == pytest.approx(L.mean(), abs=1e-3)
+    assert orc.tree_reward(tree, p, agg=orc.AGG_MAX)["r"] == L.max()
+    assert orc.tree_reward(tree, p, agg=orc.AGG_MEAN)["r"] == pytest.approx(L.mean())
+    for eta in (0.5, 1.0, 3.0):
+        r = orc.tree_reward(tree, p, eta=eta)["r"]
+        assert L.max() <= r <= L.max() + np.log(len(L)) / eta + 1e-12
+        assert r == pytest.approx(logsumexp(eta * L) / eta)
+
+
+def test_reduced_vocabulary_map_is_used_for_the_gather():
+    rng = np.random.default_rng(3)
+    D, k, g, Vd, Vt = 3, 2, 5, 4, 9
+    d2t = np.array([1, 4, 6, 8])
+    draft = rng.normal(size=(D, k, Vd))
+    target = rng.normal(size=(1 + (D - 1) * k, Vt))
+    tree = orc.build_tree(draft, D, k, g)
+    p, lse_t = orc.target_node_probs(tree, target, d2t)
+    for n in range(g):
+        r = int(tree.ctx_row[n])
+        assert p[n] == pytest.approx(softmax(target[r])[d2t[tree.token[n]]])
+    assert np.all(np.isnan(lse_t) == ~np.isin(np.arange(target.shape[0]), tree.ctx_row))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_greedy_path_length_is_max_L_for_one_hot_targets(seed):
+    """App. A case (b): at temperature 0 each L_i is the common-prefix length with
+    the greedy target trajectory and the accepted length is max_i L_i."""
+    rng = np.random.default_rng(50 + seed)
+    D, k, g, V = 4, 3, 14, 8
+    draft = rng.normal(size=(D, k, V)) * 2
+    tree = orc.build_tree(draft, D, k, g)
+    R = 1 + (D - 1) * k
+    greedy = rng.integers(0, V, size=R)
+    # make the target agree with the draft's best token on most rows so paths are long
+    for r in range(R):
+        d, j = (0, 0) if r == 0 else (1 + (r - 1) // k, (r - 1) % k)
+        if rng.random() < 0.8:
+            greedy[r] = int(np.argsort(-draft[d, j])[rng.integers(0, 2)])
+    target = np.full((R, V), -1000.0)
+    target[np.arange(R), greedy] = 1000.0
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    L = rw["Lc"][rw["leaves"]]
+    path = orc.longest_accepted(tree, target)
+    assert np.allclose(L, np.round(L))
+    assert len(path["nodes"]) == int(round(L.max()))
+    # the path is parent-linked with depths 1..l and the reported rows are the contexts
+    for j, n in enumerate(path["nodes"]):
+        assert tree.depth[n] == j + 1
+        assert tree.parent[n] == (path["nodes"][j - 1] if j else -1)
+        assert path["rows"][j] == tree.ctx_row[n]
+        assert greedy[path["rows"][j]] == tree.token[n]
+        assert path["logp"][j] == tree.logp[n]
+
+
+def test_walk_stops_at_unexpanded_node_and_on_mismatch():
+    D, k, V = 3, 2, 4
+    draft = np.zeros((D, k, V))
+    draft[0, 0] = [5, 4, 0, 0]
+    draft[1, 0] = [0, 0, 5, 4]
+    draft[1, 1] = [-9, -9, -9, -9.5]
+    draft[2, 0] = [1, 0, 0, 0]
+    draft[2, 1] = [1, 0, 0, 0]
+    tree = orc.build_tree(draft, D, k, 4)
+    target = np.zeros((1 + (D - 1) * k, V))
+    target[0, 0] = 9        # accepts token 0 at depth 1
+    target[1, 3] = 9        # greedy token 3 under slot 0: child (token 3) selected?
+    path = orc.longest_accepted(tree, target)
+    toks = [int(tree.token[n]) for n in path["nodes"]]
+    assert toks[0] == 0
+    assert all(tree.parent[b] == a for a, b in zip(path["nodes"], path["nodes"][1:]))
+    target[0] = 0
+    target[0, 2] = 9        # greedy token not among the root's children
+    assert orc.longest_accepted(tree, target)["nodes"] == []
