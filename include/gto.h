@@ -1,0 +1,161 @@
+/*
+ * gto.h - C ABI of the B200 draft-tree pass of Group Tree Optimization (GTO).
+ *
+ * One training micro-batch holds B positions.  For every position there are G = 2
+ * draft trees: t = 0 built from the current draft model's logits, t = 1 from the
+ * frozen reference draft's.  Logit rows are inputs (one V-wide row per context):
+ *
+ *   draft  [G, B, D, k, V_draft]   row [t,b,0,0,:] is the root context; row [t,b,d,j,:]
+ *                                  (1 <= d < D) is the context reached through frontier
+ *                                  slot j of depth d; rows [t,b,0,1..k-1,:] are never read.
+ *   target [G, B, R, V_target]     R = 1 + (D-1)*k; row 0 = root context, row
+ *                                  1 + (d-1)*k + j = frontier slot j of depth d.
+ *
+ * Logits are bf16 or fp32, row-major, contiguous; V_draft and V_target must make a row a
+ * multiple of 16 bytes.  All pointers in the structs below are DEVICE pointers owned by
+ * the caller, 16-byte aligned, dense row-major with the shapes given.  The library
+ * allocates device memory only in gto_create (its workspace) and keeps no caller pointer
+ * after a call returns.  Calls enqueue work on `stream` (a cudaStream_t passed as void*)
+ * and return without synchronising; argument errors are returned at once and launch
+ * nothing.  Data faults (a non-finite row sum, a bounded wait that ran out) are recorded
+ * in a device status word read by gto_device_status.  A context is not thread-safe;
+ * use one per host thread and device.  No entry point writes to stdout or throws.
+ */
+#ifndef GTO_H_
+#define GTO_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gto_ctx gto_ctx; /* opaque; owns the workspace only */
+
+typedef enum {
+  GTO_OK = 0,
+  GTO_ERR_INVALID_ARG = 1, /* null pointer, bad shape, misaligned pointer               */
+  GTO_ERR_UNSUPPORTED = 2, /* shape outside the compiled limits (see gto_create)        */
+  GTO_ERR_WORKSPACE = 3,   /* workspace allocation failed                                */
+  GTO_ERR_CUDA = 4,        /* a CUDA runtime call failed                                 */
+  GTO_ERR_NONFINITE = 5,   /* device status: a row's log-sum-exp was not finite          */
+  GTO_ERR_TIMEOUT = 6      /* device status: a bounded wait inside a kernel ran out      */
+} gto_status;
+
+typedef enum { GTO_F32 = 0, GTO_BF16 = 1 } gto_dtype;
+
+/* Reward aggregation over the tree's sequences: Eq. 5 (log-sum-exp smooth max, the
+ * default) or the two alternatives of the aggregation ablation in Sec. 4.2. */
+typedef enum { GTO_AGG_LSE = 0, GTO_AGG_MAX = 1, GTO_AGG_MEAN = 2 } gto_agg;
+
+enum {
+  GTO_FLAG_STD_UNBIASED = 1u, /* Eq. 10 with the sample std (divide by m-1)             */
+  GTO_FLAG_NO_DEBIAS = 2u     /* Eq. 9 switched off: R_i = r(T_i) (debiasing ablation)  */
+};
+
+typedef struct {
+  int32_t B;        /* positions; a multiple of m                                       */
+  int32_t G;        /* trees per position; must be 2                                    */
+  int32_t D;        /* maximum tree depth d of Sec. 3.1                                 */
+  int32_t k;        /* top-k per node expansion and per layer (App. B: 10)              */
+  int32_t g;        /* nodes kept by the global prune, root excluded (App. B: 60)       */
+  int32_t m;        /* group size of Eq. 6 (App. B: 8); groups are consecutive positions */
+  int32_t V_draft;  /* draft vocabulary                                                  */
+  int32_t V_target; /* target vocabulary                                                 */
+  int32_t logit_dtype; /* gto_dtype of draft, target and grad                           */
+  int32_t reward_agg;  /* gto_agg                                                       */
+  float eta;        /* smooth-max temperature of Eq. 5 (App. B: 1)                      */
+  float clip_eps;   /* epsilon of Eq. 12                                                */
+  float std_delta;  /* delta of Eq. 10                                                  */
+  float grad_scale; /* factor on the summed group losses (a trainer passes omega / K)   */
+  uint32_t flags;
+} gto_config;
+
+/* The pruned draft trees (Sec. 3.1, tree policy G).  Node lists hold g nodes per tree in
+ * ascending pool index (depth-major candidate number), so a parent precedes its children. */
+typedef struct {
+  int32_t* node_token;   /* [G,B,g] draft-vocabulary id                                  */
+  int32_t* node_parent;  /* [G,B,g] list position of the parent, -1 = child of the root  */
+  int32_t* node_depth;   /* [G,B,g] 1..D                                                 */
+  int32_t* node_ctx_row; /* [G,B,g] context row (0..R-1) the token was proposed from     */
+  int32_t* node_slot;    /* [G,B,g] frontier slot of the node at its depth, -1 = not expanded */
+  int32_t* node_pool;    /* [G,B,g] pool index: c at depth 1, k + (d-2)k^2 + j*k + c later */
+  float* node_logp;      /* [G,B,g] draft log-probability of the edge into the node      */
+  double* node_score;    /* [G,B,g] global acceptance score: sum of node_logp on the path */
+  uint64_t* node_mask;   /* [G,B,g,W] W = ceil(g/64): bit a of row n = a is n or an ancestor */
+  double* row_lse;       /* [G,B,R] log-sum-exp of every draft context row               */
+} gto_tree;
+
+/* Draft Tree Reward (Eq. 3-5) and the longest accepted sequence (Sec. 3.2) of tree 0. */
+typedef struct {
+  double* reward;        /* [G,B] r = R(T; eta)                                          */
+  double* etree;         /* [G,B] sum over nodes of the path product (exact expected
+                                  accepted tokens under target sampling; auxiliary)      */
+  int32_t* n_leaves;     /* [G,B] number N of sequences (leaves) in Eq. 5                */
+  float* node_ptarget;   /* [G,B,g] target probability of the node's token in its context */
+  float* node_pathprod;  /* [G,B,g] Eq. 4: product of node_ptarget from the root         */
+  float* node_L;         /* [G,B,g] Eq. 3 for the sequence ending at the node            */
+  double* row_lse_t;     /* [G,B,R] target log-sum-exp; NaN for rows no node uses        */
+  int32_t* row_argmax_t; /* [G,B,R] greedy target token (lowest id on ties); -1 likewise */
+  int32_t* path_len;     /* [B] l_i: accepted draft tokens of tree 0 under the greedy target */
+  int32_t* path_node;    /* [B,D] list positions of the accepted nodes; -1 beyond l_i    */
+  int32_t* path_row;     /* [B,D] context row of each step (the draft row that produced it) */
+  int32_t* path_token;   /* [B,D] draft token ids                                        */
+  float* path_logp;      /* [B,D] draft log-probability of each step; 0 beyond l_i       */
+} gto_reward;
+
+/* Group statistics and surrogate of Eq. 9-12. */
+typedef struct {
+  double* R;        /* [B] debiased reward, Eq. 9                                        */
+  double* adv;      /* [B] standardised advantage, Eq. 10                                */
+  double* ratio;    /* [B] s_i of Eq. 11                                                 */
+  double* coeff;    /* [B] factor on (onehot - softmax) for every step of position i     */
+  int32_t* active;  /* [B] 1 if the unclipped branch of Eq. 12 is the minimum            */
+  double* loss;     /* [B/m] group losses of Eq. 12                                      */
+} gto_grad_stats;
+
+/* Validates the configuration and allocates the workspace on `device`.
+ * Limits: G == 2; 1 <= k and k*k <= 128; 1 <= g <= min(128, k + (D-1)k^2); 1 <= D <= 16;
+ * B % m == 0; k <= V_draft; V * sizeof(logit) a multiple of 16 for both vocabularies.
+ * Returns GTO_ERR_UNSUPPORTED outside them. */
+gto_status gto_create(gto_ctx** ctx, const gto_config* cfg, int device);
+gto_status gto_destroy(gto_ctx* ctx);
+
+/* Tree policy G of Sec. 3.1 for all G*B trees: per context row the draft log-softmax and
+ * its k best tokens (value descending, id ascending); layer-wise expansion keeping the k
+ * best of the k*k candidates of each layer by cumulative log-probability (Fig. 1 caption:
+ * path confidence is the product of edge probabilities); global top-g over all
+ * k + (D-1)k^2 candidates.  Every tie goes to the lower index.  Writes every array of *out. */
+gto_status gto_build_tree(gto_ctx* ctx, const void* draft_logits, const gto_tree* out,
+                          void* stream);
+
+/* Draft Tree Reward, Eq. 3-5, and the longest accepted sequence of Sec. 3.2.  Reads only
+ * the target rows that are the context of a selected node.  d2t maps draft ids to target
+ * ids ([V_draft] int32, device, injective); NULL means identity and needs
+ * V_draft == V_target.  Writes every array of *out. */
+gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* target_logits,
+                           const int32_t* d2t, const gto_reward* out, void* stream);
+
+/* Eq. 9-12 and the derivative of the summed group losses with respect to the draft logits:
+ * grad[b,j,:] = coeff_b * (onehot(path_token[b,j]) - softmax(draft row path_row[b,j] of
+ * tree 0)) for j < path_len[b], zero otherwise (also when the ratio is clipped).
+ * old_logp [B,D] fp32: log-probabilities of the accepted tokens under the old / reference
+ * draft (entries beyond path_len ignored).  grad [B,D,V_draft] in the logit dtype. */
+gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft_logits,
+                                    const gto_tree* tree, const gto_reward* reward,
+                                    const float* old_logp, void* grad,
+                                    const gto_grad_stats* out, void* stream);
+
+/* Synchronises `stream`, then reads and clears the device status word:
+ * *host_code = GTO_OK, GTO_ERR_NONFINITE or GTO_ERR_TIMEOUT. */
+gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code);
+
+/* Number of kernel launches the library has enqueued through this context. */
+int64_t gto_launch_count(const gto_ctx* ctx);
+
+const char* gto_status_string(gto_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GTO_H_ */

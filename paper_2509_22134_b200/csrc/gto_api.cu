@@ -1,0 +1,261 @@
+// C ABI of the GTO draft-tree pass: argument validation, workspace, launch sequencing.
+#include <new>
+
+#include "gto_common.cuh"
+#include "gto_internal.h"
+
+struct gto_ctx {
+  gto_config cfg;
+  int device;
+  int R, P;
+  char* ws;           // one allocation
+  int32_t* top_id;    // [G*B*R, k] draft row top-k ids
+  float* top_z;       // [G*B*R, k] draft row top-k logits
+  int32_t* list;      // [G*B*R] needed target rows
+  int32_t* list_count;
+  int32_t* status;
+  int64_t launches;
+};
+
+namespace {
+
+size_t align_up(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    ok = cudaGetDevice(&prev) == cudaSuccess && cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+template <typename S>
+bool all_set(const S* s) {
+  // every member of the output structs is a pointer
+  const void* const* p = reinterpret_cast<const void* const*>(s);
+  for (size_t i = 0; i < sizeof(S) / sizeof(void*); ++i)
+    if (p[i] == nullptr || !aligned16(p[i])) return false;
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* gto_status_string(gto_status s) {
+  switch (s) {
+    case GTO_OK: return "ok";
+    case GTO_ERR_INVALID_ARG: return "invalid argument";
+    case GTO_ERR_UNSUPPORTED: return "shape outside the compiled limits";
+    case GTO_ERR_WORKSPACE: return "workspace allocation failed";
+    case GTO_ERR_CUDA: return "CUDA runtime error";
+    case GTO_ERR_NONFINITE: return "non-finite logit row";
+    case GTO_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
+  if (!out || !c) return GTO_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (c->B <= 0 || c->D <= 0 || c->k <= 0 || c->g <= 0 || c->m <= 0 || c->V_draft <= 0 ||
+      c->V_target <= 0)
+    return GTO_ERR_INVALID_ARG;
+  if (c->logit_dtype != GTO_F32 && c->logit_dtype != GTO_BF16) return GTO_ERR_INVALID_ARG;
+  if (c->reward_agg < GTO_AGG_LSE || c->reward_agg > GTO_AGG_MEAN) return GTO_ERR_INVALID_ARG;
+  if (!(c->eta > 0.f) || !(c->clip_eps >= 0.f) || !(c->std_delta >= 0.f))
+    return GTO_ERR_INVALID_ARG;
+  if (c->B % c->m != 0) return GTO_ERR_INVALID_ARG;
+  if (c->k > c->V_draft) return GTO_ERR_INVALID_ARG;
+  const int64_t P = c->k + static_cast<int64_t>(c->D - 1) * c->k * c->k;
+  if (c->g > P) return GTO_ERR_INVALID_ARG;
+  if (c->G != 2) return GTO_ERR_UNSUPPORTED;
+  if (c->k > gto::kMaxTopK || c->k * c->k > gto::kMaxLayer || c->g > gto::kMaxNodes ||
+      c->D > gto::kMaxDepth)
+    return GTO_ERR_UNSUPPORTED;
+  const int eb = c->logit_dtype == GTO_BF16 ? 2 : 4;
+  if ((static_cast<int64_t>(c->V_draft) * eb) % 16 || (static_cast<int64_t>(c->V_target) * eb) % 16)
+    return GTO_ERR_UNSUPPORTED;
+  const int R = 1 + (c->D - 1) * c->k;
+  const int64_t rows = static_cast<int64_t>(c->G) * c->B * R;
+  if (rows >= (1ll << 31) / c->k) return GTO_ERR_UNSUPPORTED;
+
+  DeviceGuard guard(device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  gto_ctx* ctx = new (std::nothrow) gto_ctx();
+  if (!ctx) return GTO_ERR_WORKSPACE;
+  ctx->cfg = *c;
+  ctx->device = device;
+  ctx->R = R;
+  ctx->P = static_cast<int>(P);
+  ctx->launches = 0;
+  size_t off = 0;
+  const size_t o_id = off;  off += align_up(rows * c->k * sizeof(int32_t));
+  const size_t o_z = off;   off += align_up(rows * c->k * sizeof(float));
+  const size_t o_list = off; off += align_up(rows * sizeof(int32_t));
+  const size_t o_cnt = off; off += 256;
+  const size_t o_st = off;  off += 256;
+  if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return GTO_ERR_WORKSPACE;
+  }
+  ctx->top_id = reinterpret_cast<int32_t*>(ctx->ws + o_id);
+  ctx->top_z = reinterpret_cast<float*>(ctx->ws + o_z);
+  ctx->list = reinterpret_cast<int32_t*>(ctx->ws + o_list);
+  ctx->list_count = reinterpret_cast<int32_t*>(ctx->ws + o_cnt);
+  ctx->status = reinterpret_cast<int32_t*>(ctx->ws + o_st);
+  if (cudaMemset(ctx->ws + o_cnt, 0, 512) != cudaSuccess) {
+    cudaFree(ctx->ws);
+    delete ctx;
+    return GTO_ERR_CUDA;
+  }
+  *out = ctx;
+  return GTO_OK;
+}
+
+gto_status gto_destroy(gto_ctx* ctx) {
+  if (!ctx) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaFree(ctx->ws);
+  delete ctx;
+  return e == cudaSuccess ? GTO_OK : GTO_ERR_CUDA;
+}
+
+gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, void* stream) {
+  if (!ctx || !draft || !out || !aligned16(draft) || !all_set(out)) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  const gto_config& c = ctx->cfg;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  gto::RowReduceArgs r{};
+  r.logits = draft;
+  r.dtype = c.logit_dtype;
+  r.V = c.V_draft;
+  r.R = ctx->R;
+  r.pad = c.k - 1;
+  r.list = nullptr;
+  r.list_count = nullptr;
+  r.n_rows = c.G * c.B * ctx->R;
+  r.k = c.k;
+  r.out_lse = out->row_lse;
+  r.out_id = ctx->top_id;
+  r.out_z = ctx->top_z;
+  r.status = ctx->status;
+  if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  gto::TreeBuildArgs t{};
+  t.n_trees = c.G * c.B;
+  t.D = c.D;
+  t.k = c.k;
+  t.g = c.g;
+  t.R = ctx->R;
+  t.row_lse = out->row_lse;
+  t.top_id = ctx->top_id;
+  t.top_z = ctx->top_z;
+  t.out = *out;
+  if (gto::launch_tree_build(t, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  return GTO_OK;
+}
+
+gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* target,
+                           const int32_t* d2t, const gto_reward* out, void* stream) {
+  if (!ctx || !tree || !target || !out || !aligned16(target) || !all_set(tree) || !all_set(out))
+    return GTO_ERR_INVALID_ARG;
+  const gto_config& c = ctx->cfg;
+  if (!d2t && c.V_draft != c.V_target) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int n_trees = c.G * c.B;
+  gto::RewardPlanArgs p{};
+  p.n_trees = n_trees;
+  p.g = c.g;
+  p.R = ctx->R;
+  p.node_ctx_row = tree->node_ctx_row;
+  p.list = ctx->list;
+  p.list_count = ctx->list_count;
+  p.row_lse_t = out->row_lse_t;
+  p.row_argmax_t = out->row_argmax_t;
+  if (gto::launch_reward_plan(p, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  gto::RowReduceArgs r{};
+  r.logits = target;
+  r.dtype = c.logit_dtype;
+  r.V = c.V_target;
+  r.R = ctx->R;
+  r.pad = 0;
+  r.list = ctx->list;
+  r.list_count = ctx->list_count;
+  r.n_rows = n_trees * ctx->R;
+  r.k = 1;
+  r.out_lse = out->row_lse_t;
+  r.out_id = out->row_argmax_t;
+  r.out_z = nullptr;
+  r.status = ctx->status;
+  if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  gto::RewardArgs w{};
+  w.B = c.B; w.G = c.G; w.D = c.D; w.k = c.k; w.g = c.g; w.R = ctx->R;
+  w.V_target = c.V_target;
+  w.dtype = c.logit_dtype;
+  w.agg = c.reward_agg;
+  w.eta = c.eta;
+  w.target = target;
+  w.d2t = d2t;
+  w.tree = *tree;
+  w.out = *out;
+  if (gto::launch_tree_reward(w, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  return GTO_OK;
+}
+
+gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_tree* tree,
+                                    const gto_reward* reward, const float* old_logp, void* grad,
+                                    const gto_grad_stats* out, void* stream) {
+  if (!ctx || !draft || !tree || !reward || !old_logp || !grad || !out || !aligned16(draft) ||
+      !aligned16(grad) || !aligned16(old_logp) || !all_set(tree) || !all_set(reward) ||
+      !all_set(out))
+    return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  const gto_config& c = ctx->cfg;
+  gto::GradArgs a{};
+  a.B = c.B; a.D = c.D; a.k = c.k; a.R = ctx->R; a.m = c.m; a.V = c.V_draft;
+  a.dtype = c.logit_dtype;
+  a.clip_eps = c.clip_eps;
+  a.std_delta = c.std_delta;
+  a.grad_scale = c.grad_scale;
+  a.flags = c.flags;
+  a.draft = draft;
+  a.row_lse = tree->row_lse;
+  a.reward = *reward;
+  a.old_logp = old_logp;
+  a.grad = grad;
+  a.out = *out;
+  if (gto::launch_surrogate_grad(a, static_cast<cudaStream_t>(stream), &ctx->launches) !=
+      cudaSuccess)
+    return GTO_ERR_CUDA;
+  return GTO_OK;
+}
+
+gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code) {
+  if (!ctx || !host_code) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t word = 0;
+  if (cudaMemcpyAsync(&word, ctx->status, sizeof(word), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+      cudaMemsetAsync(ctx->status, 0, sizeof(word), s) != cudaSuccess ||
+      cudaStreamSynchronize(s) != cudaSuccess)
+    return GTO_ERR_CUDA;
+  *host_code = (word & gto::kStatusTimeout)     ? GTO_ERR_TIMEOUT
+               : (word & gto::kStatusNonFinite) ? GTO_ERR_NONFINITE
+                                                : GTO_OK;
+  return GTO_OK;
+}
+
+int64_t gto_launch_count(const gto_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+"""Runs the CUDA library on a synthetic workload and checks it against the oracle.
+
+Shared by the GPU parity tests and the smoke check.  The only place where the product
+package and the oracle meet.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import check as ocheck
+from paper_2509_22134_b200 import synth
+from paper_2509_22134_b200.runner import GtoPass
+
+
+def gather_outputs(p: GtoPass, pos):
+    """Library outputs restricted to the positions `pos`, as numpy arrays."""
+    idx = torch.as_tensor(pos, device=p.device, dtype=torch.long)
+    out = {}
+    for name, t in p.tree.items():
+        out[name] = t.index_select(1, idx).cpu().numpy()
+    for name, t in p.reward.items():
+        dim = 0 if name.startswith("path_") else 1
+        out[name] = t.index_select(dim, idx).cpu().numpy()
+    for name, t in p.stats.items():
+        if name == "loss":
+            groups = sorted(set(int(b) // p.w.m for b in pos))
+            out[name] = t[torch.as_tensor(groups, device=p.device)].cpu().numpy()
+        else:
+            out[name] = t.index_select(0, idx).cpu().numpy()
+    out["grad"] = p.grad.index_select(0, idx).float().cpu().numpy().astype(np.float64)
+    return out
+
+
+def run_pass(w: synth.Workload, device="cuda:0", data=None, **kw):
+    if data is None:
+        data = synth.generate(w, device)
+    p = GtoPass(w, device, **kw)
+    p.build_tree(data["draft"])
+    p.tree_reward(data["target"], data["d2t"])
+    p.set_old_logp_from_path()
+    p.surrogate_grad(data["draft"])
+    assert p.status() == 0, "device status word set"
+    return p, data
+
+
+def check_against_oracle(w: synth.Workload, p: GtoPass, data, groups, cfg_extra=None):
+    """Oracle comparison on the listed groups (each m consecutive positions)."""
+    pos = [gidx * w.m + i for gidx in groups for i in range(w.m)]
+    idx = torch.as_tensor(pos, device=p.device, dtype=torch.long)
+    draft = data["draft"].index_select(1, idx).float().cpu().numpy()
+    target = data["target"].index_select(1, idx).float().cpu().numpy()
+    d2t = None if data["d2t"] is None else data["d2t"].cpu().numpy().astype(np.int64)
+    gpu = gather_outputs(p, pos)
+
+    class Cfg:
+        pass
+    cfg = Cfg()
+    for name in ("B", "G", "D", "k", "g", "m", "eta", "clip_eps", "std_delta", "grad_scale"):
+        setattr(cfg, name, getattr(w, name))
+    for key, val in (cfg_extra or {}).items():
+        setattr(cfg, key, val)
+
+    def old_fn(path_logp, path_row, path_token, path_len, positions):
+        out = np.zeros_like(path_logp)
+        for j, b in enumerate(positions):
+            out[j] = synth.old_logp_from_path(w, path_logp[j:j + 1], path_row[j:j + 1],
+                                              path_token[j:j + 1], path_len[j:j + 1], b0=b)[0]
+        return out
+
+    return ocheck.check_positions(cfg, draft, target, d2t, gpu, old_fn, pos)

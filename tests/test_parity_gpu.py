@@ -1,0 +1,125 @@
+"""GPU parity: the CUDA library against the oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2509_22134_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def harness():
+    import harness as h
+    return h
+
+
+def test_config0_all_positions(harness):
+    w = synth.WORKLOADS[0]
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=[0])
+    assert rep["near_tie_trees"] == 0
+    print(rep)
+
+
+@pytest.mark.parametrize("V,D,k,g,B,dtype", [
+    (4104, 4, 3, 17, 16, "bf16"),     # ragged tail: 4104 = 16*256 + 8
+    (1000, 5, 10, 60, 8, "f32"),
+    (16, 3, 4, 12, 8, "f32"),         # fewer vectors than threads
+    (33000, 2, 10, 60, 8, "bf16"),
+    (2048, 7, 11, 128, 8, "bf16"),    # compiled limits: k*k = 121, g = 128
+    (512, 1, 8, 5, 8, "f32"),         # depth 1: the root row only
+])
+def test_small_shapes(harness, V, D, k, g, B, dtype):
+    w = synth.Workload("t", B=B, V_draft=V, V_target=V, D=D, k=k, g=g, dtype=dtype, seed=V + D)
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=list(range(B // w.m)))
+    print(rep)
+
+
+def test_reduced_draft_vocabulary(harness):
+    w = synth.Workload("t", B=16, V_draft=2048, V_target=8200, D=4, k=5, g=30, seed=77)
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=[0, 1])
+    print(rep)
+
+
+def test_massive_ties_take_the_exact_path(harness):
+    """Constant and two-valued rows: every candidate ties; ids must follow the index."""
+    w = synth.Workload("t", B=8, V_draft=4096, V_target=4096, D=3, k=4, g=12, dtype="bf16", seed=5)
+    data = synth.generate(w, DEV)
+    data["draft"].zero_()
+    data["draft"][:, 1::2, :, :, 100:] = -1.0
+    data["target"].zero_()
+    p, data = harness.run_pass(w, DEV, data=data)
+    rep = harness.check_against_oracle(w, p, data, groups=[0])
+    print(rep)
+
+
+def test_variants_max_mean_unbiased_nodebias(harness):
+    from oracle import gto_oracle as orc
+    from paper_2509_22134_b200 import binding as gto
+    w = synth.Workload("t", B=16, V_draft=1024, V_target=1024, D=4, k=4, g=20, seed=9)
+    for agg, oagg in ((gto.GTO_AGG_MAX, orc.AGG_MAX), (gto.GTO_AGG_MEAN, orc.AGG_MEAN)):
+        p, data = harness.run_pass(w, DEV, reward_agg=agg)
+        harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(agg=oagg))
+    p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_STD_UNBIASED | gto.GTO_FLAG_NO_DEBIAS)
+    harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(unbiased=True, debias=False))
+
+
+def test_deterministic_integer_outputs(harness):
+    w = synth.WORKLOADS[1].with_B(32)
+    p1, data = harness.run_pass(w, DEV)
+    p2, _ = harness.run_pass(w, DEV, data=data)
+    for name in ("node_token", "node_parent", "node_pool", "node_mask"):
+        assert torch.equal(p1.tree[name], p2.tree[name])
+    assert torch.equal(p1.reward["path_node"], p2.reward["path_node"])
+    assert torch.equal(p1.tree["node_score"], p2.tree["node_score"])
+    assert torch.equal(p1.grad, p2.grad)
+
+
+def test_nonfinite_row_sets_status_and_bad_args_are_refused(harness):
+    from paper_2509_22134_b200 import binding as gto
+    w = synth.WORKLOADS[0]
+    data = synth.generate(w, DEV)
+    data["draft"][0, 3, 1, 2, 17] = float("nan")
+    from paper_2509_22134_b200.runner import GtoPass
+    p = GtoPass(w, DEV)
+    p.build_tree(data["draft"])
+    assert p.status() == 5          # GTO_ERR_NONFINITE
+    assert p.status() == 0          # cleared by the read
+    with pytest.raises(gto.GtoError):
+        gto.gto_tree_reward(p.ctx, p.tree, data["target"].view(-1)[1:], None, p.reward)   # misaligned
+    cfg = gto.make_config(8, 3, 4, 12, 3, 512, 512, "f32")     # B % m != 0
+    with pytest.raises(gto.GtoError):
+        gto.gto_create(cfg, 0)
+    cfg = gto.make_config(8, 3, 4, 12, 8, 510, 512, "bf16")    # row not a multiple of 16 bytes
+    with pytest.raises(gto.GtoError):
+        gto.gto_create(cfg, 0)
+
+
+@pytest.mark.parametrize("cfg_id,groups", [(1, [0, 31, 63]), (2, [0, 127]), (3, [0, 63]), (4, [0, 255])])
+def test_baseline_configs_sampled_groups(harness, cfg_id, groups):
+    """The full-size workloads in the launch configuration the benchmark times; the oracle
+    checks whole groups sampled from the ends of the batch."""
+    w = synth.WORKLOADS[cfg_id]
+    free, _ = torch.cuda.mem_get_info()
+    need = (w.G * w.B * w.D * w.k * w.V_draft + w.G * w.B * w.R * w.V_target + w.B * w.D * w.V_draft) * 2
+    if free < need * 1.1 + (4 << 30):
+        pytest.skip("not enough free device memory for this workload")
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=groups)
+    print(cfg_id, rep)
+    # every tree obeys the structural invariants, at any size
+    par = p.tree["node_parent"]
+    n = torch.arange(w.g, device=par.device)
+    assert bool((par < n).all()) and bool((par >= -1).all())
+    assert bool((p.tree["node_pool"][..., 1:] > p.tree["node_pool"][..., :-1]).all())
+    assert bool((p.reward["path_len"] >= 0).all()) and bool((p.reward["path_len"] <= w.D).all())
+    assert bool(torch.isfinite(p.reward["reward"]).all())
+    A = p.stats["adv"].view(-1, w.m)
+    assert float(A.sum(dim=1).abs().max()) < 1e-6
+    del p, data
+    torch.cuda.empty_cache()
