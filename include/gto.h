@@ -153,6 +153,27 @@ gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code);
 /* Number of kernel launches the library has enqueued through this context. */
 int64_t gto_launch_count(const gto_ctx* ctx);
 
+/* Kernels of one pass, in launch order (index into the arrays of gto_kernel_times). */
+enum {
+  GTO_K_DRAFT_ROWS = 0,  /* Sec. 3.1 (i): log-softmax + top-k of every draft row          */
+  GTO_K_TREE_BUILD = 1,  /* Sec. 3.1 (i)-(ii): layer-wise expansion, global top-g         */
+  GTO_K_REWARD_PLAN = 2, /* list of target rows that are the context of a selected node   */
+  GTO_K_TARGET_ROWS = 3, /* Eq. 4: log-sum-exp and greedy token of every listed target row */
+  GTO_K_TREE_REWARD = 4, /* Eq. 3-5 and the longest accepted sequence                      */
+  GTO_K_GROUP_STATS = 5, /* Eq. 9-12 per group                                             */
+  GTO_K_GRAD_ROWS = 6,   /* derivative of Eq. 12 into the draft rows of the accepted path  */
+  GTO_K_COUNT = 7
+};
+
+/* Per-kernel device timing, off by default.  While enabled, every launch is bracketed by
+ * two CUDA events on the caller's stream (host memory only; no device allocation). */
+gto_status gto_kernel_timing(gto_ctx* ctx, int enable);
+
+/* Synchronises `stream`, adds up the recorded launches since the last call and clears the
+ * record: total_ms[i] = summed device time of kernel i, launches[i] = how many.  Both
+ * arrays are HOST arrays of GTO_K_COUNT entries. */
+gto_status gto_kernel_times(gto_ctx* ctx, void* stream, double* total_ms, int64_t* launches);
+
 const char* gto_status_string(gto_status s);
 
 #ifdef __cplusplus

@@ -373,3 +373,43 @@ def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE)
         rewards.append(rw)
     path = longest_accepted(trees[0], target_b[0], d2t)
     return dict(trees=trees, rewards=rewards, path=path)
+
+
+def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, agg=AGG_LSE,
+               delta=1e-6, eps=0.2, grad_scale=1.0, unbiased=False, debias=True):
+    """The whole pass of Algorithm 1's inner loop on ONE group of m positions: trees and
+    rewards of both drafts, the longest accepted sequences, Eq. 9-12 and the gradient rows.
+    Sequences the functions above; adds no arithmetic of its own.
+
+    draft_g: [G, m, D, k, V_d], target_g: [G, m, R, V_t].
+    old_logp_fn(path_logp[m,D], path_row[m,D], path_token[m,D], path_len[m]) -> [m, D]:
+    the old-policy log-probabilities of the accepted tokens (an input of the method).
+    Returns dict(fwd, R, A, path_len, path_logp, path_row, path_token, old, sur, grad[m,D,V_d]).
+    """
+    V = draft_g.shape[-1]
+    fwd = [position_forward(np.asarray(draft_g[:, i], dtype=np.float64),
+                            np.asarray(target_g[:, i], dtype=np.float64), D, k, g, d2t, eta, agg)
+           for i in range(m)]
+    r_cur = np.array([f["rewards"][0]["r"] for f in fwd])
+    r_ref = np.array([f["rewards"][1]["r"] for f in fwd])
+    R, A = group_advantages(r_cur, r_ref, m, delta, unbiased=unbiased, debias=debias)
+    path_len = np.array([len(f["path"]["nodes"]) for f in fwd])
+    path_logp = np.zeros((m, D))
+    path_row = np.full((m, D), -1, dtype=np.int64)
+    path_tok = np.full((m, D), -1, dtype=np.int64)
+    for i, f in enumerate(fwd):
+        l = path_len[i]
+        path_logp[i, :l] = f["path"]["logp"]
+        path_row[i, :l] = f["path"]["rows"]
+        path_tok[i, :l] = f["path"]["tokens"]
+    old = old_logp_fn(path_logp, path_row, path_tok, path_len)
+    sur = clipped_surrogate(path_logp, old, path_len, A, m, eps, grad_scale)
+    grad = np.zeros((m, D, V))
+    for i, f in enumerate(fwd):
+        l = path_len[i]
+        d_i = np.asarray(draft_g[0, i], dtype=np.float64).reshape(D * k, V)
+        rows = [d_i[0 if r == 0 else k + r - 1] for r in path_row[i, :l]]
+        lse = [f["trees"][0].row_lse[r] for r in path_row[i, :l]]
+        grad[i] = surrogate_grad_rows(rows, lse, list(path_tok[i, :l]), sur["coeff"][i], D, V)
+    return dict(fwd=fwd, R=R, A=A, path_len=path_len, path_logp=path_logp, path_row=path_row,
+                path_token=path_tok, old=old, sur=sur, grad=grad)

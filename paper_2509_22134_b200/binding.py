@@ -66,10 +66,12 @@ _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ct
 _lib.gto_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_int32)]
 _lib.gto_launch_count.argtypes = [_vp]
 _lib.gto_launch_count.restype = ctypes.c_int64
+_lib.gto_kernel_timing.argtypes = [_vp, ctypes.c_int]
+_lib.gto_kernel_times.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
 _lib.gto_status_string.argtypes = [ctypes.c_int]
 _lib.gto_status_string.restype = ctypes.c_char_p
 for _f in ("gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
-           "gto_group_surrogate_grad", "gto_device_status"):
+           "gto_group_surrogate_grad", "gto_device_status", "gto_kernel_timing", "gto_kernel_times"):
     getattr(_lib, _f).restype = ctypes.c_int
 
 
@@ -181,5 +183,23 @@ def gto_launch_count(ctx: int) -> int:
     return int(_lib.gto_launch_count(ctx))
 
 
+KERNEL_NAMES = ["draft_rows", "tree_build", "reward_plan", "target_rows", "tree_reward",
+                "group_stats", "grad_rows"]   # GTO_K_* order
+
+
+def gto_kernel_timing(ctx: int, enable: bool):
+    _check(_lib.gto_kernel_timing(ctx, int(bool(enable))), "gto_kernel_timing")
+
+
+def gto_kernel_times(ctx: int, stream=None) -> dict:
+    """{kernel name: (total device ms, launches)} since the last call; synchronises."""
+    n = len(KERNEL_NAMES)
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_int64 * n)()
+    _check(_lib.gto_kernel_times(ctx, _stream_ptr(stream), ms, cnt), "gto_kernel_times")
+    return {name: (ms[i], cnt[i]) for i, name in enumerate(KERNEL_NAMES)}
+
+
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
-           "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string"]
+           "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
+           "gto_kernel_timing", "gto_kernel_times"]

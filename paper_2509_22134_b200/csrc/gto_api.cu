@@ -1,5 +1,6 @@
 // C ABI of the GTO draft-tree pass: argument validation, workspace, launch sequencing.
 #include <new>
+#include <vector>
 
 #include "gto_common.cuh"
 #include "gto_internal.h"
@@ -15,6 +16,10 @@ struct gto_ctx {
   int32_t* list_count;
   int32_t* status;
   int64_t launches;
+  bool timing;
+  struct Span { cudaEvent_t t0, t1; int kernel; };
+  std::vector<Span> spans;   // event pairs, reused across reads
+  size_t spans_used;
 };
 
 namespace {
@@ -31,6 +36,27 @@ struct DeviceGuard {
   }
   ~DeviceGuard() {
     if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+// Brackets one kernel launch with two events when per-kernel timing is on.
+struct LaunchSpan {
+  gto_ctx* c;
+  cudaStream_t s;
+  gto_ctx::Span* span = nullptr;
+  LaunchSpan(gto_ctx* ctx, int kernel, cudaStream_t stream) : c(ctx), s(stream) {
+    if (!c->timing) return;
+    if (c->spans_used == c->spans.size()) {
+      gto_ctx::Span n{};
+      if (cudaEventCreate(&n.t0) != cudaSuccess || cudaEventCreate(&n.t1) != cudaSuccess) return;
+      c->spans.push_back(n);
+    }
+    span = &c->spans[c->spans_used++];
+    span->kernel = kernel;
+    cudaEventRecord(span->t0, s);
+  }
+  ~LaunchSpan() {
+    if (span) cudaEventRecord(span->t1, s);
   }
 };
 
@@ -94,6 +120,8 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->R = R;
   ctx->P = static_cast<int>(P);
   ctx->launches = 0;
+  ctx->timing = false;
+  ctx->spans_used = 0;
   size_t off = 0;
   const size_t o_id = off;  off += align_up(rows * c->k * sizeof(int32_t));
   const size_t o_z = off;   off += align_up(rows * c->k * sizeof(float));
@@ -122,6 +150,10 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
 gto_status gto_destroy(gto_ctx* ctx) {
   if (!ctx) return GTO_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
+  for (auto& sp : ctx->spans) {
+    cudaEventDestroy(sp.t0);
+    cudaEventDestroy(sp.t1);
+  }
   cudaError_t e = cudaFree(ctx->ws);
   delete ctx;
   return e == cudaSuccess ? GTO_OK : GTO_ERR_CUDA;
@@ -147,7 +179,10 @@ gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, 
   r.out_id = ctx->top_id;
   r.out_z = ctx->top_z;
   r.status = ctx->status;
-  if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  {
+    LaunchSpan span(ctx, GTO_K_DRAFT_ROWS, s);
+    if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  }
   gto::TreeBuildArgs t{};
   t.n_trees = c.G * c.B;
   t.D = c.D;
@@ -158,6 +193,7 @@ gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, 
   t.top_id = ctx->top_id;
   t.top_z = ctx->top_z;
   t.out = *out;
+  LaunchSpan span(ctx, GTO_K_TREE_BUILD, s);
   if (gto::launch_tree_build(t, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;
 }
@@ -181,7 +217,10 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   p.list_count = ctx->list_count;
   p.row_lse_t = out->row_lse_t;
   p.row_argmax_t = out->row_argmax_t;
-  if (gto::launch_reward_plan(p, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  {
+    LaunchSpan span(ctx, GTO_K_REWARD_PLAN, s);
+    if (gto::launch_reward_plan(p, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  }
   gto::RowReduceArgs r{};
   r.logits = target;
   r.dtype = c.logit_dtype;
@@ -196,7 +235,10 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   r.out_id = out->row_argmax_t;
   r.out_z = nullptr;
   r.status = ctx->status;
-  if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  {
+    LaunchSpan span(ctx, GTO_K_TARGET_ROWS, s);
+    if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  }
   gto::RewardArgs w{};
   w.B = c.B; w.G = c.G; w.D = c.D; w.k = c.k; w.g = c.g; w.R = ctx->R;
   w.V_target = c.V_target;
@@ -207,6 +249,7 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   w.d2t = d2t;
   w.tree = *tree;
   w.out = *out;
+  LaunchSpan span(ctx, GTO_K_TREE_REWARD, s);
   if (gto::launch_tree_reward(w, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;
 }
@@ -234,9 +277,13 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
   a.old_logp = old_logp;
   a.grad = grad;
   a.out = *out;
-  if (gto::launch_surrogate_grad(a, static_cast<cudaStream_t>(stream), &ctx->launches) !=
-      cudaSuccess)
-    return GTO_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  {
+    LaunchSpan span(ctx, GTO_K_GROUP_STATS, s);
+    if (gto::launch_group_stats(a, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  }
+  LaunchSpan span(ctx, GTO_K_GRAD_ROWS, s);
+  if (gto::launch_grad_rows(a, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;
 }
 
@@ -257,5 +304,35 @@ gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code) {
 }
 
 int64_t gto_launch_count(const gto_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+gto_status gto_kernel_timing(gto_ctx* ctx, int enable) {
+  if (!ctx) return GTO_ERR_INVALID_ARG;
+  ctx->timing = enable != 0;
+  return GTO_OK;
+}
+
+gto_status gto_kernel_times(gto_ctx* ctx, void* stream, double* total_ms, int64_t* launches) {
+  if (!ctx || !total_ms || !launches) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return GTO_ERR_CUDA;
+  for (int i = 0; i < GTO_K_COUNT; ++i) {
+    total_ms[i] = 0.0;
+    launches[i] = 0;
+  }
+  gto_status st = GTO_OK;
+  for (size_t i = 0; i < ctx->spans_used; ++i) {
+    const gto_ctx::Span& sp = ctx->spans[i];
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, sp.t0, sp.t1) != cudaSuccess) {
+      st = GTO_ERR_CUDA;
+      continue;
+    }
+    total_ms[sp.kernel] += ms;
+    ++launches[sp.kernel];
+  }
+  ctx->spans_used = 0;
+  return st;
+}
 
 }  // extern "C"

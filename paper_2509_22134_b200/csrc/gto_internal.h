@@ -71,6 +71,7 @@ struct GradArgs {
   void* grad;
   gto_grad_stats out;
 };
-cudaError_t launch_surrogate_grad(const GradArgs& a, cudaStream_t stream, int64_t* launches);
+cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* launches);
+cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches);
 
 }  // namespace gto

@@ -3,13 +3,23 @@
 // with k = 1, the target rows (log-sum-exp for the probabilities of Eq. 4 and the greedy
 // target token).  One CTA per row; every logit byte is read once from HBM.
 //
+// Log-sum-exp: a warp sums 2^(z*log2e - ref) against ONE reference, log2e times the largest
+// of the first logits it loads (a sample of ~1000, so the reference sits close to the row
+// maximum and the terms that dominate the sum have small arguments).  Partial sums are
+// plain additions; the warps' sums are shifted to a common reference and combined in fp64,
+// and lse = ref / log2e + ln2 * log2(sum), so the fp32 rounding of log2e cancels for the
+// dominant terms.  A row in which some warp's maximum lies more than kRefHeadroom (log2
+// units) above its reference is summed again against the row maximum (rare: re-reads it).
+//
 // Selection without sorting: while streaming, each thread keeps only the running maximum
-// of its own elements.  The k-th largest of the thread maxima is a lower bound tau of the
-// row's k-th largest value (those maxima are k distinct elements), so the row's top-k are
-// among the elements >= tau, and only threads whose maximum reaches tau can hold any.
-// Those few threads rescan their own vectors (L2 hits) and push (value, id) candidates;
-// one warp then extracts the k best keys exactly.  A row with more candidates than the
-// buffer holds (massive ties) takes k exact arg-max rounds over the row instead.
+// of its own elements.  From every warp's two largest thread maxima (k <= 8: the largest)
+// the k-th largest is a lower bound tau of the row's k-th largest value (they are distinct
+// elements), so the row's top-k are among the elements >= tau, and only threads whose
+// maximum reaches tau can hold any.  The warp of such a thread rescans that thread's
+// vectors cooperatively (L2 hits, one round trip) and pushes (value, id) candidates; each
+// candidate's rank among the candidates is then counted directly.  With k = 1 the first
+// vector holding the thread maximum is remembered, so no rescan is needed.  A row with
+// more candidates than the buffer holds (massive ties) takes k exact arg-max rounds.
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
@@ -20,36 +30,53 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / kWarp;
 constexpr int kUnroll = 4;
 constexpr int kCandCap = 1024;
+constexpr float kRefHeadroom = 64.f;  // 2^64 * V stays far inside fp32 range
+
+static_assert(kMaxTopK <= 2 * kWarps, "tau needs k distinct thread maxima from 2 per warp");
 
 struct RowSmem {
-  float warp_top[kWarps][kMaxTopK];  // each warp's k largest thread maxima, descending
-  float warp_ref[kWarps];            // log2-domain reference of the warp's partial sum
+  float warp_top[2 * kWarps];  // each warp's two largest thread maxima
   float warp_sum[kWarps];
-  float tau;
+  float warp_ref[kWarps];
+  int warp_bad[kWarps];  // the warp's reference was too far below its maximum
   int n_cand;
-  float cand_z[kCandCap];
-  int cand_id[kCandCap];
+  unsigned long long cand[kCandCap];  // (value, id) keys
   unsigned long long round_best[kWarps];
   unsigned long long prev_key;
 };
 
-// Descending bitonic sort of one value per lane.
-__device__ __forceinline__ float warp_sort_desc(float v, int lane) {
+template <typename T>
+__device__ __forceinline__ void push_candidates(RowSmem& sm, const uint4& v, int vec_index,
+                                                float tau) {
+  constexpr int E = T::kPerVec;
+  float f[E];
+  T::unpack(v, f);
 #pragma unroll
-  for (int k2 = 2; k2 <= 32; k2 <<= 1) {
-#pragma unroll
-    for (int j = k2 >> 1; j > 0; j >>= 1) {
-      float o = __shfl_xor_sync(kFull, v, j);
-      bool desc = (lane & k2) == 0;
-      bool lower = (lane & j) == 0;
-      v = (lower == desc) ? fmaxf(v, o) : fminf(v, o);
+  for (int e = 0; e < E; ++e) {
+    if (f[e] >= tau) {
+      int slot = atomicAdd(&sm.n_cand, 1);
+      if (slot < kCandCap) sm.cand[slot] = make_key(f[e], vec_index * E + e);
     }
   }
-  return v;
+}
+
+// Sum of 2^(z*log2e - ref) over the thread's share of the row (used by the rare second pass).
+template <typename T>
+__device__ __forceinline__ float thread_sum(const char* row, int nvec, int tid, float ref) {
+  constexpr int E = T::kPerVec;
+  float s = 0.f;
+  for (int i = tid; i < nvec; i += kThreads) {
+    uint4 v = ld_stream16(row + static_cast<size_t>(i) * 16);
+    float f[E];
+    T::unpack(v, f);
+#pragma unroll
+    for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, -ref));
+  }
+  return s;
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads) row_reduce_kernel(RowReduceArgs a) {
+__global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a) {
   constexpr int E = T::kPerVec;
   __shared__ RowSmem sm;
   const int tid = threadIdx.x;
@@ -68,10 +95,11 @@ __global__ void __launch_bounds__(kThreads) row_reduce_kernel(RowReduceArgs a) {
   const int nvec = a.V / E;
   const int k = a.k;
 
-  // ---- pass 1: per-thread running maximum and sum of 2^(z*log2e - ref)
-  float m = -INFINITY, ref = -INFINITY, s = 0.f;
-  for (int i0 = tid; i0 < nvec; i0 += kThreads * kUnroll) {
-    uint4 v[kUnroll];
+  // ---- pass 1: per-thread maximum (and the first vector holding it) and exponential sum
+  float ref = 0.f, ref_max = -INFINITY;
+  float m = -INFINITY, s = 0.f;
+  int best_i = tid;
+  auto load_batch = [&](uint4(&v)[kUnroll], int i0) {
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       int i = i0 + u * kThreads;
@@ -79,89 +107,117 @@ __global__ void __launch_bounds__(kThreads) row_reduce_kernel(RowReduceArgs a) {
                         : make_uint4(T::kNegInfWord, T::kNegInfWord, T::kNegInfWord,
                                      T::kNegInfWord);
     }
+  };
+  auto consume = [&](const uint4& vec, int i) {
+    float f[E];
+    T::unpack(vec, f);
+    float vmax = f[0];
+#pragma unroll
+    for (int e = 1; e < E; ++e) vmax = fmaxf(vmax, f[e]);
+    if (vmax > m) {
+      m = vmax;
+      best_i = i;
+    }
+    // pairwise sum of the vector's terms, then one add into the running sum
+#pragma unroll
+    for (int e = 0; e < E; ++e) f[e] = ex2_approx(fmaf(f[e], kLog2e, -ref));
+#pragma unroll
+    for (int w = 1; w < E; w <<= 1) {
+#pragma unroll
+      for (int e = 0; e < E; e += 2 * w) f[e] += f[e + w];
+    }
+    s += f[0];
+  };
+  {
+    // first batch: its largest logit across the warp fixes the warp's reference
+    uint4 v[kUnroll];
+    load_batch(v, tid);
+    float bmax = -INFINITY;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       float f[E];
       T::unpack(v[u], f);
-      float vmax = f[0];
 #pragma unroll
-      for (int e = 1; e < E; ++e) vmax = fmaxf(vmax, f[e]);
-      if (vmax > m) {
-        float nref = vmax * kLog2e;
-        s *= ex2_approx(ref - nref);
-        m = vmax;
-        ref = nref;
-      }
-#pragma unroll
-      for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, -ref));
+      for (int e = 0; e < E; ++e) bmax = fmaxf(bmax, f[e]);
     }
+    ref_max = warp_max_f32(bmax);
+    ref = ref_max == -INFINITY ? 0.f : ref_max * kLog2e;
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) consume(v[u], tid + u * kThreads);
+  }
+  for (int i0 = tid + kThreads * kUnroll; i0 < nvec; i0 += kThreads * kUnroll) {
+    uint4 v[kUnroll];
+    load_batch(v, i0);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) consume(v[u], i0 + u * kThreads);
   }
 
-  // ---- warp level: k largest thread maxima, and the warp's partial sum
+  // ---- warp level: two largest thread maxima, partial sum
   {
-    float sorted = warp_sort_desc(m, lane);
-    if (lane < k) sm.warp_top[warp][lane] = sorted;
-    float wref = warp_max_f32(ref);
-    float part = (ref == -INFINITY) ? 0.f : s * ex2_approx(ref - wref);
-    part = warp_sum_f32(part);
+    float m1 = warp_max_f32(m);
+    unsigned holders = __ballot_sync(kFull, m == m1);
+    float rest = (lane == __ffs(holders) - 1) ? -INFINITY : m;
+    float m2 = warp_max_f32(rest);
+    float part = warp_sum_f32(s);
     if (lane == 0) {
-      sm.warp_ref[warp] = wref;
+      sm.warp_top[2 * warp] = m1;
+      sm.warp_top[2 * warp + 1] = m2;
       sm.warp_sum[warp] = part;
+      sm.warp_ref[warp] = ref;
+      // a warp without data has m1 = -inf and no terms; NaN or -inf references fail the test
+      sm.warp_bad[warp] = (m1 != -INFINITY && !((m1 - ref_max) * kLog2e <= kRefHeadroom)) ? 1 : 0;
     }
   }
   if (tid == 0) sm.n_cand = 0;
   __syncthreads();
 
-  // ---- warp 0: tau = k-th largest thread maximum (with multiplicity)
-  if (warp == 0) {
-    constexpr int kPer = (kWarps * kMaxTopK + 31) / 32;
-    float mine[kPer];
-#pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-      int idx = lane + q * 32;
-      int w = idx / kMaxTopK, c = idx % kMaxTopK;
-      mine[q] = (w < kWarps && c < k) ? sm.warp_top[w][c] : -INFINITY;
+  // ---- tau: the k-th largest of the warps' top maxima (every warp computes it)
+  float tau, row_max;
+  {
+    const int per = (k <= kWarps) ? 1 : 2;  // entries taken from each warp
+    const int n = per * kWarps;
+    float mine = -INFINITY;
+    int my_slot = 0;
+    if (lane < n) {
+      my_slot = (per == 1) ? 2 * lane : lane;
+      mine = sm.warp_top[my_slot];
     }
-    float tau = -INFINITY;
-    for (int round = 0; round < k; ++round) {
-      float best = mine[0];
-#pragma unroll
-      for (int q = 1; q < kPer; ++q) best = fmaxf(best, mine[q]);
-      float wbest = warp_max_f32(best);
-      tau = wbest;
-      unsigned holders = __ballot_sync(kFull, best == wbest);
-      if (lane == __ffs(holders) - 1) {  // drop one instance
-        bool done = false;
-#pragma unroll
-        for (int q = 0; q < kPer; ++q) {
-          if (!done && mine[q] == wbest) {
-            mine[q] = -INFINITY;
-            done = true;
-          }
-        }
-      }
+    int rank = 0;
+    for (int j = 0; j < n; ++j) {
+      int slot = (per == 1) ? 2 * j : j;
+      float o = sm.warp_top[slot];
+      rank += (o > mine || (o == mine && slot < my_slot)) ? 1 : 0;
     }
-    if (lane == 0) sm.tau = tau;
+    unsigned hit = __ballot_sync(kFull, lane < n && rank == k - 1);
+    tau = __shfl_sync(kFull, mine, __ffs(hit) - 1);
+    row_max = warp_max_f32(mine);
   }
-  __syncthreads();
-  const float tau = sm.tau;
 
-  // ---- pass 2: threads that can hold a top-k element rescan their own vectors
-  if (m >= tau) {
-    for (int i = tid; i < nvec; i += kThreads) {
-      uint4 v = ld_stream16(row + static_cast<size_t>(i) * 16);
-      float f[E];
-      T::unpack(v, f);
+  // ---- rare: a reference was too low -> sum again against the row maximum
+  int resum = 0;
 #pragma unroll
-      for (int e = 0; e < E; ++e) {
-        if (f[e] >= tau) {
-          int slot = atomicAdd(&sm.n_cand, 1);
-          if (slot < kCandCap) {
-            sm.cand_z[slot] = f[e];
-            sm.cand_id[slot] = i * E + e;
-          }
-        }
-      }
+  for (int w = 0; w < kWarps; ++w) resum |= sm.warp_bad[w];
+  if (resum) {
+    ref = row_max * kLog2e;
+    float part = warp_sum_f32(thread_sum<T>(row, nvec, tid, ref));
+    if (lane == 0) {
+      sm.warp_sum[warp] = part;
+      sm.warp_ref[warp] = ref;
+    }
+  }
+
+  // ---- candidates: every element >= tau
+  if (k == 1) {
+    // the first vector holding the thread maximum is known; ties keep the lowest index
+    if (m >= tau) push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(best_i) * 16),
+                                     best_i, tau);
+  } else {
+    unsigned todo = __ballot_sync(kFull, m >= tau);
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      for (int i = warp * 32 + src + lane * kThreads; i < nvec; i += 32 * kThreads)
+        push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(i) * 16), i, tau);
     }
   }
   __syncthreads();
@@ -171,21 +227,14 @@ __global__ void __launch_bounds__(kThreads) row_reduce_kernel(RowReduceArgs a) {
   float* out_z = a.out_z ? a.out_z + static_cast<size_t>(gid) * k : nullptr;
 
   if (n_cand <= kCandCap) {
-    // ---- exact top-k among the candidates: k rounds of warp arg-max on (value, id) keys
-    if (warp == 0) {
-      uint64_t prev = ~0ull;
-      for (int round = 0; round < k; ++round) {
-        uint64_t best = 0;
-        for (int c = lane; c < n_cand; c += 32) {
-          uint64_t key = make_key(sm.cand_z[c], sm.cand_id[c]);
-          if (key < prev && key > best) best = key;
-        }
-        best = warp_max_u64(best);
-        prev = best;
-        if (lane == 0) {
-          out_id[round] = key_id(best);
-          if (out_z) out_z[round] = key_value(best);
-        }
+    // ---- exact top-k among the candidates: a candidate's rank is the number of larger keys
+    for (int c = tid; c < n_cand; c += kThreads) {
+      const uint64_t key = sm.cand[c];
+      int rank = 0;
+      for (int j = 0; j < n_cand; ++j) rank += sm.cand[j] > key ? 1 : 0;
+      if (rank < k) {
+        out_id[rank] = key_id(key);
+        if (out_z) out_z[rank] = key_value(key);
       }
     }
   } else {
@@ -219,17 +268,17 @@ __global__ void __launch_bounds__(kThreads) row_reduce_kernel(RowReduceArgs a) {
     }
   }
 
-  // ---- row log-sum-exp: combine the warps in fp64
+  // ---- row log-sum-exp: shift the warps' sums to a common reference, combine in fp64
   if (tid == 0) {
-    float Ref = sm.warp_ref[0];
-    for (int w = 1; w < kWarps; ++w) Ref = fmaxf(Ref, sm.warp_ref[w]);
+    float Ref = -INFINITY;
+    for (int w = 0; w < kWarps; ++w)
+      if (sm.warp_sum[w] != 0.f) Ref = fmaxf(Ref, sm.warp_ref[w]);
     double S = 0.0;
-    for (int w = 0; w < kWarps; ++w) {
-      if (sm.warp_ref[w] != -INFINITY)
+    for (int w = 0; w < kWarps; ++w)
+      if (sm.warp_sum[w] != 0.f)
         S += static_cast<double>(sm.warp_sum[w]) *
              exp2(static_cast<double>(sm.warp_ref[w]) - static_cast<double>(Ref));
-    }
-    double lse = (static_cast<double>(Ref) + log2(S)) * kLn2;
+    double lse = static_cast<double>(Ref) / static_cast<double>(kLog2e) + kLn2 * log2(S);
     if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
     a.out_lse[gid] = lse;
   }

@@ -116,12 +116,14 @@ __global__ void __launch_bounds__(kGradThreads) grad_rows_kernel(GradArgs a) {
 
 }  // namespace
 
-cudaError_t launch_surrogate_grad(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
+cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
   int groups = a.B / a.m;
   group_stats_kernel<<<(groups + kStatWarps - 1) / kStatWarps, kStatWarps * 32, 0, stream>>>(a);
   ++*launches;
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
   int vec_per_row = a.V / (a.dtype == GTO_BF16 ? 8 : 4);
   int split = (vec_per_row + kGradThreads * 8 - 1) / (kGradThreads * 8);  // ~8 vectors/thread
   if (split < 1) split = 1;
