@@ -68,6 +68,20 @@ struct Bf16 {
   __device__ static __forceinline__ float load1(const void* base, size_t idx) {
     return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[idx]);
   }
+  // Running maximum kept as two packed bf16 lanes (4 instructions per 8 logits).
+  using MaxAcc = uint32_t;
+  __device__ static __forceinline__ MaxAcc max_init() { return kNegInfWord; }
+  __device__ static __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+  }
+  __device__ static __forceinline__ void max_update(MaxAcc& acc, const uint4& v) {
+    acc = max2(acc, max2(max2(v.x, v.y), max2(v.z, v.w)));
+  }
+  __device__ static __forceinline__ float max_value(MaxAcc acc) {
+    return fmaxf(__uint_as_float(acc << 16), __uint_as_float(acc & 0xffff0000u));
+  }
 };
 
 struct F32 {
@@ -87,6 +101,13 @@ struct F32 {
   __device__ static __forceinline__ float load1(const void* base, size_t idx) {
     return reinterpret_cast<const float*>(base)[idx];
   }
+  using MaxAcc = float;
+  __device__ static __forceinline__ MaxAcc max_init() { return -INFINITY; }
+  __device__ static __forceinline__ void max_update(MaxAcc& acc, const uint4& v) {
+    acc = fmaxf(fmaxf(acc, fmaxf(__uint_as_float(v.x), __uint_as_float(v.y))),
+                fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+  }
+  __device__ static __forceinline__ float max_value(MaxAcc acc) { return acc; }
 };
 
 // Total order on (value, id): larger key = better candidate = (value desc, id asc).
@@ -100,10 +121,12 @@ __device__ __forceinline__ uint64_t make_key(float z, int id) {
 __device__ __forceinline__ int key_id(uint64_t key) {
   return static_cast<int>(0xffffffffu - static_cast<uint32_t>(key));
 }
+// Inverse of orderable().
+__device__ __forceinline__ float from_orderable(uint32_t o) {
+  return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu));
+}
 __device__ __forceinline__ float key_value(uint64_t key) {
-  uint32_t o = static_cast<uint32_t>(key >> 32);
-  uint32_t u = o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu);
-  return __uint_as_float(u);
+  return from_orderable(static_cast<uint32_t>(key >> 32));
 }
 
 __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {

@@ -11,31 +11,48 @@
 // dominant terms.  A row in which some warp's maximum lies more than kRefHeadroom (log2
 // units) above its reference is summed again against the row maximum (rare: re-reads it).
 //
-// Selection without sorting: while streaming, each thread keeps only the running maximum
-// of its own elements.  From every warp's two largest thread maxima (k <= 8: the largest)
+// Selection without sorting: while streaming, each thread keeps only the largest and the
+// second largest of its batch maxima (a batch = kUnroll vectors loaded together) and which
+// batch held the largest.  From every warp's ceil(k / warps) largest thread maxima
 // the k-th largest is a lower bound tau of the row's k-th largest value (they are distinct
 // elements), so the row's top-k are among the elements >= tau, and only threads whose
-// maximum reaches tau can hold any.  The warp of such a thread rescans that thread's
-// vectors cooperatively (L2 hits, one round trip) and pushes (value, id) candidates; each
-// candidate's rank among the candidates is then counted directly.  With k = 1 the first
-// vector holding the thread maximum is remembered, so no rescan is needed.  A row with
-// more candidates than the buffer holds (massive ties) takes k exact arg-max rounds.
+// maximum reaches tau can hold any.  Such a thread reloads its best batch (L2 hits, one
+// round trip) and pushes (value, id) candidates; if its second-best batch reaches tau too,
+// its warp rescans all of the thread's vectors cooperatively instead.  Each candidate's
+// rank among the candidates is then counted directly.  A row with more candidates than the
+// buffer holds (massive ties) takes k exact arg-max rounds.
+//
+// The pass is bound by instruction issue as much as by HBM (one exponential per logit), so
+// the streaming loop keeps the running maximum packed (two bf16 lanes per instruction) and
+// warp maxima use the integer redux instruction on order-preserving keys.
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
 namespace gto {
 namespace {
 
-constexpr int kThreads = 256;
+#ifndef GTO_ROW_THREADS
+#define GTO_ROW_THREADS 256
+#endif
+#ifndef GTO_ROW_UNROLL
+#define GTO_ROW_UNROLL 4
+#endif
+#ifndef GTO_ROW_MIN_CTAS
+#define GTO_ROW_MIN_CTAS (2048 / GTO_ROW_THREADS)
+#endif
+constexpr int kThreads = GTO_ROW_THREADS;
 constexpr int kWarps = kThreads / kWarp;
-constexpr int kUnroll = 4;
+constexpr int kMaxPer = (kMaxTopK + kWarps - 1) / kWarps;  // thread maxima kept per warp
+constexpr int kUnroll = GTO_ROW_UNROLL;
+constexpr int kMinCtas = GTO_ROW_MIN_CTAS;  // resident CTAs per SM the register budget allows
 constexpr int kCandCap = 1024;
 constexpr float kRefHeadroom = 64.f;  // 2^64 * V stays far inside fp32 range
 
-static_assert(kMaxTopK <= 2 * kWarps, "tau needs k distinct thread maxima from 2 per warp");
+static_assert(kMaxPer * kWarps <= 32, "one lane per kept maximum");
+constexpr uint32_t kKeyNegInf = 0x007fffffu;  // orderable(-inf): stands for "no element"
 
 struct RowSmem {
-  float warp_top[2 * kWarps];  // each warp's two largest thread maxima
+  uint32_t warp_top[kMaxPer * kWarps];  // each warp's largest thread maxima, as orderable keys
   float warp_sum[kWarps];
   float warp_ref[kWarps];
   int warp_bad[kWarps];  // the warp's reference was too far below its maximum
@@ -76,7 +93,7 @@ __device__ __forceinline__ float thread_sum(const char* row, int nvec, int tid, 
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a) {
+__global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduceArgs a) {
   constexpr int E = T::kPerVec;
   __shared__ RowSmem sm;
   const int tid = threadIdx.x;
@@ -95,10 +112,11 @@ __global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a
   const int nvec = a.V / E;
   const int k = a.k;
 
-  // ---- pass 1: per-thread maximum (and the first vector holding it) and exponential sum
+  // ---- pass 1: per-thread exponential sum; largest and second-largest batch maximum
   float ref = 0.f, ref_max = -INFINITY;
-  float m = -INFINITY, s = 0.f;
-  int best_i = tid;
+  float s = 0.f;
+  float b1 = -INFINITY, b2 = -INFINITY;  // best and second-best batch maximum of the thread
+  int i1 = tid;                          // first vector of the best batch
   auto load_batch = [&](uint4(&v)[kUnroll], int i0) {
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
@@ -108,16 +126,15 @@ __global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a
                                      T::kNegInfWord);
     }
   };
-  auto consume = [&](const uint4& vec, int i) {
+  auto batch_max = [&](const uint4(&v)[kUnroll]) {
+    typename T::MaxAcc acc = T::max_init();
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) T::max_update(acc, v[u]);
+    return T::max_value(acc);
+  };
+  auto add_terms = [&](const uint4& vec) {
     float f[E];
     T::unpack(vec, f);
-    float vmax = f[0];
-#pragma unroll
-    for (int e = 1; e < E; ++e) vmax = fmaxf(vmax, f[e]);
-    if (vmax > m) {
-      m = vmax;
-      best_i = i;
-    }
     // pairwise sum of the vector's terms, then one add into the running sum
 #pragma unroll
     for (int e = 0; e < E; ++e) f[e] = ex2_approx(fmaf(f[e], kLog2e, -ref));
@@ -132,39 +149,45 @@ __global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a
     // first batch: its largest logit across the warp fixes the warp's reference
     uint4 v[kUnroll];
     load_batch(v, tid);
-    float bmax = -INFINITY;
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      float f[E];
-      T::unpack(v[u], f);
-#pragma unroll
-      for (int e = 0; e < E; ++e) bmax = fmaxf(bmax, f[e]);
-    }
-    ref_max = warp_max_f32(bmax);
+    b1 = batch_max(v);
+    ref_max = from_orderable(__reduce_max_sync(kFull, orderable(b1)));
     ref = ref_max == -INFINITY ? 0.f : ref_max * kLog2e;
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) consume(v[u], tid + u * kThreads);
+    for (int u = 0; u < kUnroll; ++u) add_terms(v[u]);
   }
   for (int i0 = tid + kThreads * kUnroll; i0 < nvec; i0 += kThreads * kUnroll) {
     uint4 v[kUnroll];
     load_batch(v, i0);
+    const float bm = batch_max(v);
+    if (bm > b1) {  // an equal maximum counts as second best: both batches then hold candidates
+      b2 = b1;
+      b1 = bm;
+      i1 = i0;
+    } else {
+      b2 = fmaxf(b2, bm);
+    }
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) consume(v[u], i0 + u * kThreads);
+    for (int u = 0; u < kUnroll; ++u) add_terms(v[u]);
   }
 
-  // ---- warp level: two largest thread maxima, partial sum
+  // ---- warp level: the warp's `per` largest thread maxima, partial sum
+  const int per = (k + kWarps - 1) / kWarps;  // per * kWarps >= k distinct elements
   {
-    float m1 = warp_max_f32(m);
-    unsigned holders = __ballot_sync(kFull, m == m1);
-    float rest = (lane == __ffs(holders) - 1) ? -INFINITY : m;
-    float m2 = warp_max_f32(rest);
-    float part = warp_sum_f32(s);
+    uint32_t key = orderable(b1);
+    uint32_t k1 = 0;
+    for (int p = 0; p < per; ++p) {
+      const uint32_t top = __reduce_max_sync(kFull, key);
+      if (p == 0) k1 = top;
+      if (lane == 0) sm.warp_top[warp * kMaxPer + p] = top;
+      const unsigned holders = __ballot_sync(kFull, key == top);
+      if (lane == __ffs(holders) - 1) key = kKeyNegInf;
+    }
+    const float part = warp_sum_f32(s);
     if (lane == 0) {
-      sm.warp_top[2 * warp] = m1;
-      sm.warp_top[2 * warp + 1] = m2;
       sm.warp_sum[warp] = part;
       sm.warp_ref[warp] = ref;
-      // a warp without data has m1 = -inf and no terms; NaN or -inf references fail the test
+      // a warp without data has maximum -inf and no terms; NaN or -inf references fail the test
+      const float m1 = from_orderable(k1);
       sm.warp_bad[warp] = (m1 != -INFINITY && !((m1 - ref_max) * kLog2e <= kRefHeadroom)) ? 1 : 0;
     }
   }
@@ -174,23 +197,16 @@ __global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a
   // ---- tau: the k-th largest of the warps' top maxima (every warp computes it)
   float tau, row_max;
   {
-    const int per = (k <= kWarps) ? 1 : 2;  // entries taken from each warp
-    const int n = per * kWarps;
-    float mine = -INFINITY;
-    int my_slot = 0;
-    if (lane < n) {
-      my_slot = (per == 1) ? 2 * lane : lane;
-      mine = sm.warp_top[my_slot];
+    uint32_t key = kKeyNegInf;
+    if (lane < per * kWarps) key = sm.warp_top[(lane / per) * kMaxPer + lane % per];
+    uint32_t top = __reduce_max_sync(kFull, key);
+    row_max = from_orderable(top);
+    for (int round = 1; round < k; ++round) {  // drop one holder of the maximum, k-1 times
+      const unsigned holders = __ballot_sync(kFull, key == top);
+      if (lane == __ffs(holders) - 1) key = kKeyNegInf;
+      top = __reduce_max_sync(kFull, key);
     }
-    int rank = 0;
-    for (int j = 0; j < n; ++j) {
-      int slot = (per == 1) ? 2 * j : j;
-      float o = sm.warp_top[slot];
-      rank += (o > mine || (o == mine && slot < my_slot)) ? 1 : 0;
-    }
-    unsigned hit = __ballot_sync(kFull, lane < n && rank == k - 1);
-    tau = __shfl_sync(kFull, mine, __ffs(hit) - 1);
-    row_max = warp_max_f32(mine);
+    tau = from_orderable(top);
   }
 
   // ---- rare: a reference was too low -> sum again against the row maximum
@@ -207,12 +223,15 @@ __global__ void __launch_bounds__(kThreads, 8) row_reduce_kernel(RowReduceArgs a
   }
 
   // ---- candidates: every element >= tau
-  if (k == 1) {
-    // the first vector holding the thread maximum is known; ties keep the lowest index
-    if (m >= tau) push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(best_i) * 16),
-                                     best_i, tau);
-  } else {
-    unsigned todo = __ballot_sync(kFull, m >= tau);
+  {
+    const bool one_batch = b1 >= tau && !(b2 >= tau);
+    if (one_batch) {  // all of the thread's candidates are in its best batch
+      uint4 v[kUnroll];
+      load_batch(v, i1);
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) push_candidates<T>(sm, v[u], i1 + u * kThreads, tau);
+    }
+    unsigned todo = __ballot_sync(kFull, b2 >= tau);  // several batches: rescan the thread
     while (todo) {
       const int src = __ffs(todo) - 1;
       todo &= todo - 1;
