@@ -194,19 +194,21 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   if (tid == 0) sm.n_cand = 0;
   __syncthreads();
 
-  // ---- tau: the k-th largest of the warps' top maxima (every warp computes it)
+  // ---- tau: the k-th largest of the warps' top maxima (every warp computes it): each lane
+  //      counts the entries that precede its own in (value desc, lane asc) order
   float tau, row_max;
   {
+    const int n = per * kWarps;
     uint32_t key = kKeyNegInf;
-    if (lane < per * kWarps) key = sm.warp_top[(lane / per) * kMaxPer + lane % per];
-    uint32_t top = __reduce_max_sync(kFull, key);
-    row_max = from_orderable(top);
-    for (int round = 1; round < k; ++round) {  // drop one holder of the maximum, k-1 times
-      const unsigned holders = __ballot_sync(kFull, key == top);
-      if (lane == __ffs(holders) - 1) key = kKeyNegInf;
-      top = __reduce_max_sync(kFull, key);
+    if (lane < n) key = sm.warp_top[(lane / per) * kMaxPer + lane % per];
+    int rank = 0;
+    for (int j = 0; j < n; ++j) {
+      const uint32_t o = __shfl_sync(kFull, key, j);
+      rank += (o > key || (o == key && j < lane)) ? 1 : 0;
     }
-    tau = from_orderable(top);
+    const unsigned hit = __ballot_sync(kFull, lane < n && rank == k - 1);
+    tau = from_orderable(__shfl_sync(kFull, key, __ffs(hit) - 1));
+    row_max = from_orderable(__reduce_max_sync(kFull, key));
   }
 
   // ---- rare: a reference was too low -> sum again against the row maximum
