@@ -112,18 +112,26 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   const int nvec = a.V / E;
   const int k = a.k;
 
-  // ---- pass 1: per-thread exponential sum; largest and second-largest batch maximum
+  // ---- pass 1: per-thread exponential sum; largest and second-largest batch maximum.
+  //      Batches that are complete for every thread run without bounds checks.
+  constexpr int kBatchVecs = kThreads * kUnroll;
+  const int nfull = nvec / kBatchVecs;
+  const bool ragged = nfull * kBatchVecs < nvec;
+  const uint4* p = reinterpret_cast<const uint4*>(row) + tid;
   float ref = 0.f, ref_max = -INFINITY;
   float s = 0.f;
   float b1 = -INFINITY, b2 = -INFINITY;  // best and second-best batch maximum of the thread
-  int i1 = tid;                          // first vector of the best batch
-  auto load_batch = [&](uint4(&v)[kUnroll], int i0) {
+  int i1 = 0;                            // batch that held the best
+  auto load_full = [&](uint4(&v)[kUnroll], const uint4* q) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) v[u] = ld_stream16(q + u * kThreads);
+  };
+  auto load_checked = [&](uint4(&v)[kUnroll], int b) {
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
-      int i = i0 + u * kThreads;
-      v[u] = (i < nvec) ? ld_stream16(row + static_cast<size_t>(i) * 16)
-                        : make_uint4(T::kNegInfWord, T::kNegInfWord, T::kNegInfWord,
-                                     T::kNegInfWord);
+      const int i = tid + b * kBatchVecs + u * kThreads;
+      v[u] = make_uint4(T::kNegInfWord, T::kNegInfWord, T::kNegInfWord, T::kNegInfWord);
+      if (i < nvec) v[u] = ld_stream16(reinterpret_cast<const uint4*>(row) + i);
     }
   };
   auto batch_max = [&](const uint4(&v)[kUnroll]) {
@@ -132,42 +140,52 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     for (int u = 0; u < kUnroll; ++u) T::max_update(acc, v[u]);
     return T::max_value(acc);
   };
-  auto add_terms = [&](const uint4& vec) {
-    float f[E];
-    T::unpack(vec, f);
-    // pairwise sum of the vector's terms, then one add into the running sum
+  auto add_terms = [&](const uint4(&v)[kUnroll]) {
 #pragma unroll
-    for (int e = 0; e < E; ++e) f[e] = ex2_approx(fmaf(f[e], kLog2e, -ref));
+    for (int u = 0; u < kUnroll; ++u) {
+      float f[E];
+      T::unpack(v[u], f);
+      // pairwise sum of the vector's terms, then one add into the running sum
 #pragma unroll
-    for (int w = 1; w < E; w <<= 1) {
+      for (int e = 0; e < E; ++e) f[e] = ex2_approx(fmaf(f[e], kLog2e, -ref));
 #pragma unroll
-      for (int e = 0; e < E; e += 2 * w) f[e] += f[e + w];
+      for (int w = 1; w < E; w <<= 1) {
+#pragma unroll
+        for (int e = 0; e < E; e += 2 * w) f[e] += f[e + w];
+      }
+      s += f[0];
     }
-    s += f[0];
+  };
+  auto track = [&](float bm, int b) {
+    if (bm > b1) {  // an equal maximum counts as second best: both batches then hold candidates
+      b2 = b1;
+      b1 = bm;
+      i1 = b;
+    } else {
+      b2 = fmaxf(b2, bm);
+    }
   };
   {
     // first batch: its largest logit across the warp fixes the warp's reference
     uint4 v[kUnroll];
-    load_batch(v, tid);
+    if (nfull > 0) load_full(v, p); else load_checked(v, 0);
     b1 = batch_max(v);
     ref_max = from_orderable(__reduce_max_sync(kFull, orderable(b1)));
     ref = ref_max == -INFINITY ? 0.f : ref_max * kLog2e;
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) add_terms(v[u]);
+    add_terms(v);
   }
-  for (int i0 = tid + kThreads * kUnroll; i0 < nvec; i0 += kThreads * kUnroll) {
+  for (int b = 1; b < nfull; ++b) {
+    p += kBatchVecs;
     uint4 v[kUnroll];
-    load_batch(v, i0);
-    const float bm = batch_max(v);
-    if (bm > b1) {  // an equal maximum counts as second best: both batches then hold candidates
-      b2 = b1;
-      b1 = bm;
-      i1 = i0;
-    } else {
-      b2 = fmaxf(b2, bm);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) add_terms(v[u]);
+    load_full(v, p);
+    track(batch_max(v), b);
+    add_terms(v);
+  }
+  if (ragged && nfull > 0) {
+    uint4 v[kUnroll];
+    load_checked(v, nfull);
+    track(batch_max(v), nfull);
+    add_terms(v);
   }
 
   // ---- warp level: the warp's `per` largest thread maxima, partial sum
@@ -229,9 +247,10 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     const bool one_batch = b1 >= tau && !(b2 >= tau);
     if (one_batch) {  // all of the thread's candidates are in its best batch
       uint4 v[kUnroll];
-      load_batch(v, i1);
+      load_checked(v, i1);
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) push_candidates<T>(sm, v[u], i1 + u * kThreads, tau);
+      for (int u = 0; u < kUnroll; ++u)
+        push_candidates<T>(sm, v[u], tid + i1 * kBatchVecs + u * kThreads, tau);
     }
     unsigned todo = __ballot_sync(kFull, b2 >= tau);  // several batches: rescan the thread
     while (todo) {
