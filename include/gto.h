@@ -116,7 +116,7 @@ typedef struct {
 
 /* Validates the configuration and allocates the workspace on `device`.
  * Limits: G == 2; 1 <= k and k*k <= 128; 1 <= g <= min(128, k + (D-1)k^2); 1 <= D <= 16;
- * B % m == 0; k <= V_draft; V * sizeof(logit) a multiple of 16 for both vocabularies.
+ * B % m == 0; G*B <= 65535; k <= V_draft; V * sizeof(logit) a multiple of 16 for both vocabularies.
  * Returns GTO_ERR_UNSUPPORTED outside them. */
 gto_status gto_create(gto_ctx** ctx, const gto_config* cfg, int device);
 gto_status gto_destroy(gto_ctx* ctx);

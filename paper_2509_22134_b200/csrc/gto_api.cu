@@ -110,6 +110,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   const int R = 1 + (c->D - 1) * c->k;
   const int64_t rows = static_cast<int64_t>(c->G) * c->B * R;
   if (rows >= (1ll << 31) / c->k) return GTO_ERR_UNSUPPORTED;
+  if (static_cast<int64_t>(c->G) * c->B > 65535) return GTO_ERR_UNSUPPORTED;  // grid.y = trees
 
   DeviceGuard guard(device);
   if (!guard.ok) return GTO_ERR_CUDA;

@@ -56,6 +56,9 @@ struct RowSmem {
   float warp_sum[kWarps];
   float warp_ref[kWarps];
   int warp_bad[kWarps];  // the warp's reference was too far below its maximum
+  float tau;             // lower bound of the row's k-th largest value
+  float row_max;
+  int resum;             // some warp's reference was too low: sum again against row_max
   int n_cand;
   unsigned long long cand[kCandCap];  // (value, id) keys
   unsigned long long round_best[kWarps];
@@ -66,6 +69,10 @@ template <typename T>
 __device__ __forceinline__ void push_candidates(RowSmem& sm, const uint4& v, int vec_index,
                                                 float tau) {
   constexpr int E = T::kPerVec;
+  // most vectors hold no candidate: test the vector's maximum first
+  typename T::MaxAcc acc = T::max_init();
+  T::max_update(acc, v);
+  if (!(T::max_value(acc) >= tau)) return;
   float f[E];
   T::unpack(v, f);
 #pragma unroll
@@ -100,13 +107,18 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   const int lane = tid & 31;
   const int warp = tid >> 5;
 
-  int gid = blockIdx.x;
+  // rows come either from the work list (1-D grid) or as (row in tree, tree) = (x, y)
+  int gid, tree, r;
   if (a.list != nullptr) {
-    if (gid >= *a.list_count) return;
-    gid = a.list[gid];
+    if (blockIdx.x >= *a.list_count) return;
+    gid = a.list[blockIdx.x];
+    tree = a.pad != 0 ? gid / a.R : 0;  // a tensor without padding rows needs no split
+    r = gid - tree * a.R;
+  } else {
+    r = blockIdx.x;
+    tree = blockIdx.y;
+    gid = tree * a.R + r;
   }
-  const int tree = gid / a.R;
-  const int r = gid - tree * a.R;
   const char* row =
       static_cast<const char*>(a.logits) + tensor_row(tree, r, a.R, a.pad) * a.V * T::kBytes;
   const int nvec = a.V / E;
@@ -209,13 +221,12 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
       sm.warp_bad[warp] = (m1 != -INFINITY && !((m1 - ref_max) * kLog2e <= kRefHeadroom)) ? 1 : 0;
     }
   }
-  if (tid == 0) sm.n_cand = 0;
   __syncthreads();
 
-  // ---- tau: the k-th largest of the warps' top maxima (every warp computes it): each lane
-  //      counts the entries that precede its own in (value desc, lane asc) order
-  float tau, row_max;
-  {
+  // ---- warp 0: tau = the k-th largest of the warps' top maxima (each lane counts the
+  //      entries that precede its own in (value desc, lane asc) order); row maximum;
+  //      whether some reference was too low
+  if (warp == 0) {
     const int n = per * kWarps;
     uint32_t key = kKeyNegInf;
     if (lane < n) key = sm.warp_top[(lane / per) * kMaxPer + lane % per];
@@ -224,17 +235,21 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
       const uint32_t o = __shfl_sync(kFull, key, j);
       rank += (o > key || (o == key && j < lane)) ? 1 : 0;
     }
-    const unsigned hit = __ballot_sync(kFull, lane < n && rank == k - 1);
-    tau = from_orderable(__shfl_sync(kFull, key, __ffs(hit) - 1));
-    row_max = from_orderable(__reduce_max_sync(kFull, key));
+    const uint32_t top = __reduce_max_sync(kFull, key);
+    const int bad = __any_sync(kFull, lane < kWarps && sm.warp_bad[lane < kWarps ? lane : 0] != 0);
+    if (lane < n && rank == k - 1) sm.tau = from_orderable(key);
+    if (lane == 0) {
+      sm.row_max = from_orderable(top);
+      sm.resum = bad;
+      sm.n_cand = 0;
+    }
   }
+  __syncthreads();
+  const float tau = sm.tau;
 
   // ---- rare: a reference was too low -> sum again against the row maximum
-  int resum = 0;
-#pragma unroll
-  for (int w = 0; w < kWarps; ++w) resum |= sm.warp_bad[w];
-  if (resum) {
-    ref = row_max * kLog2e;
+  if (sm.resum) {  // uniform over the CTA
+    ref = sm.row_max * kLog2e;
     float part = warp_sum_f32(thread_sum<T>(row, nvec, tid, ref));
     if (lane == 0) {
       sm.warp_sum[warp] = part;
@@ -308,7 +323,9 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     }
   }
 
-  // ---- row log-sum-exp: shift the warps' sums to a common reference, combine in fp64
+  // ---- row log-sum-exp: shift the warps' sums to a common reference (exact powers of two
+  //      times sums that carry 2^-22 already), then log2 of the fp64 total as exponent +
+  //      log2f(mantissa in [1,2)), so the fp32 logarithm's error stays below 1e-7
   if (tid == 0) {
     float Ref = -INFINITY;
     for (int w = 0; w < kWarps; ++w)
@@ -317,8 +334,17 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     for (int w = 0; w < kWarps; ++w)
       if (sm.warp_sum[w] != 0.f)
         S += static_cast<double>(sm.warp_sum[w]) *
-             exp2(static_cast<double>(sm.warp_ref[w]) - static_cast<double>(Ref));
-    double lse = static_cast<double>(Ref) / static_cast<double>(kLog2e) + kLn2 * log2(S);
+             static_cast<double>(exp2f(sm.warp_ref[w] - Ref));
+    double lse;
+    if (S > 0.0 && S < 1e300) {
+      int ex;
+      const double mant = frexp(S, &ex);  // S = mant * 2^ex, mant in [0.5, 1)
+      const double lg = static_cast<double>(ex - 1) +
+                        static_cast<double>(log2f(static_cast<float>(mant * 2.0)));
+      lse = static_cast<double>(Ref) / static_cast<double>(kLog2e) + kLn2 * lg;
+    } else {
+      lse = (S == 0.0) ? -INFINITY : S;  // no terms, inf or NaN: reported below
+    }
     if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
     a.out_lse[gid] = lse;
   }
@@ -329,6 +355,10 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
 cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64_t* launches) {
   if (a.n_rows <= 0) return cudaSuccess;
   dim3 grid(a.n_rows), block(kThreads);
+  if (a.list == nullptr) {
+    if (a.n_rows % a.R != 0 || a.n_rows / a.R > 65535) return cudaErrorInvalidValue;
+    grid = dim3(a.R, a.n_rows / a.R);
+  }
   if (a.dtype == GTO_BF16)
     row_reduce_kernel<Bf16><<<grid, block, 0, stream>>>(a);
   else
