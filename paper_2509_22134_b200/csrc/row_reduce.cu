@@ -3,13 +3,15 @@
 // with k = 1, the target rows (log-sum-exp for the probabilities of Eq. 4 and the greedy
 // target token).  One CTA per row; every logit byte is read once from HBM.
 //
-// Log-sum-exp: a warp sums 2^(z*log2e - ref) against ONE reference, log2e times the largest
-// of the first logits it loads (a sample of ~1000, so the reference sits close to the row
-// maximum and the terms that dominate the sum have small arguments).  Partial sums are
-// plain additions; the warps' sums are shifted to a common reference and combined in fp64,
-// and lse = ref / log2e + ln2 * log2(sum), so the fp32 rounding of log2e cancels for the
-// dominant terms.  A row in which some warp's maximum lies more than kRefHeadroom (log2
-// units) above its reference is summed again against the row maximum (rare: re-reads it).
+// Log-sum-exp: a thread sums 2^(z*log2e - ref).  The reference starts as log2e times the
+// largest of the first logits its warp loads (a sample of ~1000, so it sits close to the row
+// maximum and all threads of a warp normally share it); a thread whose batch maximum rises
+// more than kRebase (log2 units) above its reference rescales its sum and moves the
+// reference up, so no argument exceeds kRebase: nothing can overflow, and the terms that
+// dominate the sum have small arguments, whose fp32 rounding is small.  Thread sums are
+// shifted to the warp's largest reference, the warps' sums to a common one and combined in
+// fp64, and lse = ref / log2e + ln2 * log2(sum), so the fp32 rounding of log2e cancels for
+// the dominant terms.
 //
 // Selection without sorting: while streaming, each thread keeps only the largest and the
 // second largest of its batch maxima (a batch = kUnroll vectors loaded together) and which
@@ -32,13 +34,13 @@ namespace gto {
 namespace {
 
 #ifndef GTO_ROW_THREADS
-#define GTO_ROW_THREADS 256
+#define GTO_ROW_THREADS 128
 #endif
 #ifndef GTO_ROW_UNROLL
 #define GTO_ROW_UNROLL 4
 #endif
 #ifndef GTO_ROW_MIN_CTAS
-#define GTO_ROW_MIN_CTAS (2048 / GTO_ROW_THREADS)
+#define GTO_ROW_MIN_CTAS 12  // 40 registers per thread: no spills in the streaming loop
 #endif
 constexpr int kThreads = GTO_ROW_THREADS;
 constexpr int kWarps = kThreads / kWarp;
@@ -46,7 +48,7 @@ constexpr int kMaxPer = (kMaxTopK + kWarps - 1) / kWarps;  // thread maxima kept
 constexpr int kUnroll = GTO_ROW_UNROLL;
 constexpr int kMinCtas = GTO_ROW_MIN_CTAS;  // resident CTAs per SM the register budget allows
 constexpr int kCandCap = 1024;
-constexpr float kRefHeadroom = 64.f;  // 2^64 * V stays far inside fp32 range
+constexpr float kRebase = 8.f;  // largest exponent argument before a thread moves its reference
 
 static_assert(kMaxPer * kWarps <= 32, "one lane per kept maximum");
 constexpr uint32_t kKeyNegInf = 0x007fffffu;  // orderable(-inf): stands for "no element"
@@ -55,10 +57,7 @@ struct RowSmem {
   uint32_t warp_top[kMaxPer * kWarps];  // each warp's largest thread maxima, as orderable keys
   float warp_sum[kWarps];
   float warp_ref[kWarps];
-  int warp_bad[kWarps];  // the warp's reference was too far below its maximum
-  float tau;             // lower bound of the row's k-th largest value
-  float row_max;
-  int resum;             // some warp's reference was too low: sum again against row_max
+  float tau;  // lower bound of the row's k-th largest value
   int n_cand;
   unsigned long long cand[kCandCap];  // (value, id) keys
   unsigned long long round_best[kWarps];
@@ -82,21 +81,6 @@ __device__ __forceinline__ void push_candidates(RowSmem& sm, const uint4& v, int
       if (slot < kCandCap) sm.cand[slot] = make_key(f[e], vec_index * E + e);
     }
   }
-}
-
-// Sum of 2^(z*log2e - ref) over the thread's share of the row (used by the rare second pass).
-template <typename T>
-__device__ __forceinline__ float thread_sum(const char* row, int nvec, int tid, float ref) {
-  constexpr int E = T::kPerVec;
-  float s = 0.f;
-  for (int i = tid; i < nvec; i += kThreads) {
-    uint4 v = ld_stream16(row + static_cast<size_t>(i) * 16);
-    float f[E];
-    T::unpack(v, f);
-#pragma unroll
-    for (int e = 0; e < E; ++e) s += ex2_approx(fmaf(f[e], kLog2e, -ref));
-  }
-  return s;
 }
 
 template <typename T>
@@ -130,7 +114,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   const int nfull = nvec / kBatchVecs;
   const bool ragged = nfull * kBatchVecs < nvec;
   const uint4* p = reinterpret_cast<const uint4*>(row) + tid;
-  float ref = 0.f, ref_max = -INFINITY;
+  float ref = 0.f;
   float s = 0.f;
   float b1 = -INFINITY, b2 = -INFINITY;  // best and second-best batch maximum of the thread
   int i1 = 0;                            // batch that held the best
@@ -169,6 +153,11 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     }
   };
   auto track = [&](float bm, int b) {
+    const float t = bm * kLog2e;
+    if (t > ref + kRebase) {  // rare: keep every argument below kRebase
+      s *= ex2_approx(ref - t);
+      ref = t;
+    }
     if (bm > b1) {  // an equal maximum counts as second best: both batches then hold candidates
       b2 = b1;
       b1 = bm;
@@ -182,7 +171,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
     uint4 v[kUnroll];
     if (nfull > 0) load_full(v, p); else load_checked(v, 0);
     b1 = batch_max(v);
-    ref_max = from_orderable(__reduce_max_sync(kFull, orderable(b1)));
+    const float ref_max = from_orderable(__reduce_max_sync(kFull, orderable(b1)));
     ref = ref_max == -INFINITY ? 0.f : ref_max * kLog2e;
     add_terms(v);
   }
@@ -204,28 +193,24 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   const int per = (k + kWarps - 1) / kWarps;  // per * kWarps >= k distinct elements
   {
     uint32_t key = orderable(b1);
-    uint32_t k1 = 0;
     for (int p = 0; p < per; ++p) {
       const uint32_t top = __reduce_max_sync(kFull, key);
-      if (p == 0) k1 = top;
       if (lane == 0) sm.warp_top[warp * kMaxPer + p] = top;
       const unsigned holders = __ballot_sync(kFull, key == top);
       if (lane == __ffs(holders) - 1) key = kKeyNegInf;
     }
-    const float part = warp_sum_f32(s);
+    // shift the thread sums to the warp's largest reference, then add them
+    const float wref = from_orderable(__reduce_max_sync(kFull, orderable(ref)));
+    const float part = warp_sum_f32(s * ex2_approx(ref - wref));
     if (lane == 0) {
       sm.warp_sum[warp] = part;
-      sm.warp_ref[warp] = ref;
-      // a warp without data has maximum -inf and no terms; NaN or -inf references fail the test
-      const float m1 = from_orderable(k1);
-      sm.warp_bad[warp] = (m1 != -INFINITY && !((m1 - ref_max) * kLog2e <= kRefHeadroom)) ? 1 : 0;
+      sm.warp_ref[warp] = wref;
     }
   }
   __syncthreads();
 
   // ---- warp 0: tau = the k-th largest of the warps' top maxima (each lane counts the
-  //      entries that precede its own in (value desc, lane asc) order); row maximum;
-  //      whether some reference was too low
+  //      entries that precede its own in (value desc, lane asc) order)
   if (warp == 0) {
     const int n = per * kWarps;
     uint32_t key = kKeyNegInf;
@@ -235,27 +220,11 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
       const uint32_t o = __shfl_sync(kFull, key, j);
       rank += (o > key || (o == key && j < lane)) ? 1 : 0;
     }
-    const uint32_t top = __reduce_max_sync(kFull, key);
-    const int bad = __any_sync(kFull, lane < kWarps && sm.warp_bad[lane < kWarps ? lane : 0] != 0);
     if (lane < n && rank == k - 1) sm.tau = from_orderable(key);
-    if (lane == 0) {
-      sm.row_max = from_orderable(top);
-      sm.resum = bad;
-      sm.n_cand = 0;
-    }
+    if (lane == 0) sm.n_cand = 0;
   }
   __syncthreads();
   const float tau = sm.tau;
-
-  // ---- rare: a reference was too low -> sum again against the row maximum
-  if (sm.resum) {  // uniform over the CTA
-    ref = sm.row_max * kLog2e;
-    float part = warp_sum_f32(thread_sum<T>(row, nvec, tid, ref));
-    if (lane == 0) {
-      sm.warp_sum[warp] = part;
-      sm.warp_ref[warp] = ref;
-    }
-  }
 
   // ---- candidates: every element >= tau
   {
