@@ -39,7 +39,8 @@ typedef enum {
   GTO_ERR_WORKSPACE = 3,   /* workspace allocation failed                                */
   GTO_ERR_CUDA = 4,        /* a CUDA runtime call failed                                 */
   GTO_ERR_NONFINITE = 5,   /* device status: a row's log-sum-exp was not finite          */
-  GTO_ERR_TIMEOUT = 6      /* device status: a bounded wait inside a kernel ran out      */
+  GTO_ERR_TIMEOUT = 6,     /* device status: a bounded wait inside a kernel ran out      */
+  GTO_ERR_TOO_LARGE = 7    /* gto_build_tree_noalloc: batch exceeds the fixed scratch    */
 } gto_status;
 
 typedef enum { GTO_F32 = 0, GTO_BF16 = 1 } gto_dtype;
@@ -128,6 +129,32 @@ gto_status gto_destroy(gto_ctx* ctx);
  * k + (D-1)k^2 candidates.  Every tie goes to the lower index.  Writes every array of *out. */
 gto_status gto_build_tree(gto_ctx* ctx, const void* draft_logits, const gto_tree* out,
                           void* stream);
+
+/* Largest G*B*R*k (draft context rows times top-k) gto_build_tree_noalloc accepts: its
+ * scratch is a fixed array of 8 bytes per entry (8 MiB) inside the library image. */
+#define GTO_NOALLOC_MAX_ENTRIES (1 << 20)
+
+/* gto_build_tree for callers that must not allocate device memory (no counterpart in the
+ * paper: it is an integration aid).  A trainer that routes every device byte through its own
+ * allocator, a process living inside a fixed memory budget, or a thread that cannot afford
+ * the device-wide stall an allocation may cause, cannot create a gto_ctx, because gto_create
+ * calls cudaMalloc.  This call needs no context: it takes the configuration directly and
+ * keeps the per-row top-k tables in a fixed device array that ships with the library (every
+ * GPU that loads the library holds those 8 MiB until the process ends).  It never calls
+ * cudaMalloc, cudaFree or any allocating routine.
+ *   - Computes exactly what gto_build_tree computes and writes every array of *out; only
+ *     B, G, D, k, g, V_draft and logit_dtype of *cfg are used.
+ *   - Returns GTO_ERR_TOO_LARGE when G*B*R*k > GTO_NOALLOC_MAX_ENTRIES: split the batch.
+ *   - The first call on a device looks up the array's device address (one
+ *     cudaGetSymbolAddress, cached per device); make that first call outside any stream
+ *     capture.
+ *   - All calls on a device share the one array and it keeps the last call's contents; the
+ *     call clears what it needs cleared.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, no dependency between them) race on it: order them.
+ *   - There is no status word to read back: a row with non-finite logits shows as a
+ *     non-finite entry of out->row_lse. */
+gto_status gto_build_tree_noalloc(const gto_config* cfg, int device, const void* draft_logits,
+                                  const gto_tree* out, void* stream);
 
 /* Draft Tree Reward, Eq. 3-5, and the longest accepted sequence of Sec. 3.2.  Reads only
  * the target rows that are the context of a selected node.  d2t maps draft ids to target

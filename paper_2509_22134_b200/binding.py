@@ -60,6 +60,9 @@ _vp = ctypes.c_void_p
 _lib.gto_create.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(gto_config), ctypes.c_int]
 _lib.gto_destroy.argtypes = [_vp]
 _lib.gto_build_tree.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), _vp]
+_lib.gto_build_tree_noalloc.argtypes = [ctypes.POINTER(gto_config), ctypes.c_int, _vp,
+                                        ctypes.POINTER(gto_tree), _vp]
+_lib.gto_build_tree_noalloc.restype = ctypes.c_int
 _lib.gto_tree_reward.argtypes = [_vp, ctypes.POINTER(gto_tree), _vp, _vp, ctypes.POINTER(gto_reward), _vp]
 _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ctypes.POINTER(gto_reward),
                                           _vp, _vp, ctypes.POINTER(gto_grad_stats), _vp]
@@ -150,6 +153,19 @@ def gto_build_tree(ctx: int, draft: torch.Tensor, tree: dict, stream=None):
            "gto_build_tree")
 
 
+GTO_NOALLOC_MAX_ENTRIES = 1 << 20
+
+
+def gto_build_tree_noalloc(cfg: gto_config, device: int, draft: torch.Tensor, tree: dict, stream=None):
+    """gto_build_tree without a context and without any device allocation: for callers
+    that must keep every device byte under their own allocator.  Raises GtoError(7) when
+    G*B*R*k exceeds GTO_NOALLOC_MAX_ENTRIES."""
+    assert draft.is_cuda and draft.is_contiguous()
+    t = _fill(gto_tree, _TREE_FIELDS, tree)
+    _check(_lib.gto_build_tree_noalloc(ctypes.byref(cfg), device, draft.data_ptr(), ctypes.byref(t),
+                                       _stream_ptr(stream)), "gto_build_tree_noalloc")
+
+
 def gto_tree_reward(ctx: int, tree: dict, target: torch.Tensor, d2t, reward: dict, stream=None):
     assert target.is_cuda and target.is_contiguous()
     if d2t is not None:
@@ -202,4 +218,4 @@ def gto_kernel_times(ctx: int, stream=None) -> dict:
 
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
            "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
-           "gto_kernel_timing", "gto_kernel_times"]
+           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc"]

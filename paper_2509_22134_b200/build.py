@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgto.so")
-SOURCES = ["gto_api.cu", "row_reduce.cu", "tree_build.cu", "tree_reward.cu", "surrogate_grad.cu"]
+SOURCES = ["gto_api.cu", "row_reduce.cu", "tree_build.cu", "tree_reward.cu", "surrogate_grad.cu",
+           "build_tree_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -82,6 +82,7 @@ const char* gto_status_string(gto_status s) {
     case GTO_ERR_CUDA: return "CUDA runtime error";
     case GTO_ERR_NONFINITE: return "non-finite logit row";
     case GTO_ERR_TIMEOUT: return "bounded device wait ran out";
+    case GTO_ERR_TOO_LARGE: return "batch exceeds the fixed scratch of the no-allocation call";
   }
   return "unknown status";
 }
