@@ -40,6 +40,11 @@ E2E_POSITIONS = 64          # positions per end-to-end step (host buffers of ~2.
 # entry is used only while the kernel source it was taken from is unchanged.
 NCU_TRAFFIC = {
     # kernel: (source file, sha256 of that file at capture time, bytes per row, V of the capture)
+    # from profiles/row_reduce_workload2_b64.md
+    "draft_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
+                   "9af7c0ab7759533b118e6bd7a2687fca4b0bf05d5b6a792af05b570b44e830a1", (512533248 + 8308480) / 7808, 32000),
+    "target_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
+                    "9af7c0ab7759533b118e6bd7a2687fca4b0bf05d5b6a792af05b570b44e830a1", (429916160 + 4603136) / 1673, 128256),
 }
 
 
@@ -206,6 +211,20 @@ def workload_config(w, n_gpus):
 
 
 # ---------------------------------------------------------------------------- GPU arm
+def shard_first_position(rank: int, positions_per_rank: int) -> int:
+    """Absolute index of a rank's first position: ranks own consecutive blocks of whole
+    groups, so no group straddles two GPUs and no collective is needed on the data path."""
+    return rank * positions_per_rank
+
+
+def max_over_ranks(values, world: int, device):
+    """Element-wise maximum of per-rank device timings (every rank gets the result)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
 def algorithmic_bytes(w, p):
     """Bytes the method must move per step, from the data-dependent counts of this batch."""
     e = w.elem_bytes
@@ -229,7 +248,7 @@ def run_gpu(args, w, rank, world, local_rank):
 
     dev = torch.device("cuda", local_rank)
     torch.cuda.set_device(dev)
-    b0 = rank * w.B
+    b0 = shard_first_position(rank, w.B)
     data = synth.generate(w, dev, b0=b0)
     p = GtoPass(w, dev)
     # the old-policy log-probabilities are an input of the gradient call: fix them once
@@ -267,10 +286,7 @@ def run_gpu(args, w, rank, world, local_rank):
     if e2e is None:
         e2e = {"ms": float("nan"), "positions": 0, "h2d": 0, "d2h": 0, "positions_per_step": 0, "steps": 0}
 
-    t = torch.tensor([ms, e2e["ms"]], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    ms, e2e_ms = float(t[0]), float(t[1])
+    ms, e2e_ms = max_over_ranks([ms, e2e["ms"]], world, dev)
     if rank != 0:
         return
 
