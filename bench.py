@@ -206,7 +206,8 @@ def run_reference(args, w, rank, world):
 def workload_config(w, n_gpus):
     return {"workload": w.name, "positions_per_gpu": w.B, "global_positions": w.B * n_gpus,
             "V_draft": w.V_draft, "V_target": w.V_target, "D": w.D, "top_k": w.k, "g": w.g, "G": w.G,
-            "m": w.m, "logits": w.dtype, "parallelism": f"replicas x{n_gpus} (positions sharded, no collective)",
+            "m": w.m, "logits": w.dtype, "grad": "rows that carry a gradient only (GTO_FLAG_GRAD_LIVE_ROWS)",
+            "parallelism": f"replicas x{n_gpus} (positions sharded, no collective)",
             "l2": "inputs (tens of GB) far exceed the 126 MB L2; no flush needed"}
 
 
@@ -250,7 +251,7 @@ def run_gpu(args, w, rank, world, local_rank):
     torch.cuda.set_device(dev)
     b0 = shard_first_position(rank, w.B)
     data = synth.generate(w, dev, b0=b0)
-    p = GtoPass(w, dev)
+    p = GtoPass(w, dev, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS)
     # the old-policy log-probabilities are an input of the gradient call: fix them once
     p.build_tree(data["draft"])
     p.tree_reward(data["target"], data["d2t"])
@@ -346,7 +347,8 @@ def run_e2e(args, w, dev, b0, world):
     data = synth.generate(we, dev, b0=b0)
     host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v)
             for k, v in data.items() if k in ("draft", "target")}
-    p = GtoPass(we, dev)
+    from paper_2509_22134_b200 import binding as gto
+    p = GtoPass(we, dev, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS)
     p.build_tree(data["draft"])
     p.tree_reward(data["target"], data["d2t"])
     p.set_old_logp_from_path(b0=b0)

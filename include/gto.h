@@ -51,7 +51,10 @@ typedef enum { GTO_AGG_LSE = 0, GTO_AGG_MAX = 1, GTO_AGG_MEAN = 2 } gto_agg;
 
 enum {
   GTO_FLAG_STD_UNBIASED = 1u, /* Eq. 10 with the sample std (divide by m-1)             */
-  GTO_FLAG_NO_DEBIAS = 2u     /* Eq. 9 switched off: R_i = r(T_i) (debiasing ablation)  */
+  GTO_FLAG_NO_DEBIAS = 2u,    /* Eq. 9 switched off: R_i = r(T_i) (debiasing ablation)  */
+  GTO_FLAG_GRAD_LIVE_ROWS = 4u /* gto_group_surrogate_grad writes only the rows that carry a
+                                  gradient (j < path_len[b] and coeff[b] != 0) and leaves the
+                                  rest of grad untouched, instead of filling it with zeros   */
 };
 
 typedef struct {
@@ -165,7 +168,9 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
 
 /* Eq. 9-12 and the derivative of the summed group losses with respect to the draft logits:
  * grad[b,j,:] = coeff_b * (onehot(path_token[b,j]) - softmax(draft row path_row[b,j] of
- * tree 0)) for j < path_len[b], zero otherwise (also when the ratio is clipped).
+ * tree 0)) for j < path_len[b], zero otherwise (also when the ratio is clipped).  With
+ * GTO_FLAG_GRAD_LIVE_ROWS the zero rows are not written (a trainer that scatters the rows
+ * into its logit gradient by path_row reads only the live ones).
  * old_logp [B,D] fp32: log-probabilities of the accepted tokens under the old / reference
  * draft (entries beyond path_len ignored).  grad [B,D,V_draft] in the logit dtype. */
 gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft_logits,

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libgto.so")
 GTO_OK = 0
 GTO_F32, GTO_BF16 = 0, 1
 GTO_AGG_LSE, GTO_AGG_MAX, GTO_AGG_MEAN = 0, 1, 2
-GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS = 1, 2
+GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS, GTO_FLAG_GRAD_LIVE_ROWS = 1, 2, 4
 
 if not os.path.exists(LIB_PATH):
     raise RuntimeError(

@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(kGradThreads) grad_rows_kernel(GradArgs a) {
   const int l = a.reward.path_len[b];
   const float c = static_cast<float>(a.out.coeff[b]);
   if (j >= l || c == 0.f) {
+    if (a.flags & GTO_FLAG_GRAD_LIVE_ROWS) return;  // the caller reads live rows only
     const uint4 zero = make_uint4(0, 0, 0, 0);
     for (int i = v0 + threadIdx.x; i < v1; i += kGradThreads)
       st_stream16(out + static_cast<size_t>(i) * 16, zero);

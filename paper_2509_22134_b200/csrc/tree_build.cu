@@ -1,30 +1,29 @@
 // Tree policy G of Sec. 3.1 on the per-row top-k tables: layer-wise expansion (the k best
 // of the k*k candidates of each layer by cumulative log-probability become the next
-// frontier) and the global top-g prune over all k + (D-1)k^2 candidates.  One warp per
-// tree; the rankings are register-resident bitonic networks over 128 (score, index)
-// pairs, exchanged with shuffles.  Scores are fp64 sums of (z - lse) so that a ranking
-// differs from an exact evaluation only where two scores agree to ~1e-7.
+// frontier) and the global top-g prune over all k + (D-1)k^2 candidates.  One 128-thread
+// CTA per tree, one thread per candidate of a layer.
+//
+// No sorting network: every ranking is counted.  The k children of one frontier node are
+// already in (score descending, index ascending) order, because a row's top-k is and the
+// score adds the same parent score to each.  A candidate's rank in its layer is therefore
+// its own child index plus, for every other parent, the number of that parent's children
+// ahead of it (a binary search over k entries).  The layers are kept sorted in shared
+// memory, and a candidate's global rank is its layer rank plus, for every other layer, the
+// number of entries ahead of it (a binary search again); only the first g of a layer can
+// reach the global top-g.  Ties go to the lower index everywhere: child index within a
+// parent, parent slot within a layer, layer (= depth) across layers, i.e. the pool index.
+// Scores are fp64 sums of (z - lse), so a ranking differs from an exact evaluation only
+// where two scores agree to ~1e-7.
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
 namespace gto {
 namespace {
 
-constexpr int kE = 4;                  // elements per lane
-constexpr int kN = 32 * kE;            // 128 = kMaxLayer = kMaxNodes
-constexpr int kWarpsPerCta = 4;
-constexpr uint32_t kInvalidAux = 0x7fffffffu;
-
-static_assert(kN == kMaxLayer && kN == kMaxNodes, "network size");
-
-struct Item {
-  uint64_t key;  // larger is better
-  uint32_t aux;  // smaller is better on equal keys
-};
-
-__device__ __forceinline__ bool better(const Item& a, const Item& b) {
-  return a.key > b.key || (a.key == b.key && a.aux < b.aux);
-}
+constexpr int kTreeThreads = 128;
+static_assert(kMaxLayer <= kTreeThreads, "one thread per layer candidate");
+static_assert(kMaxNodes <= kTreeThreads, "one thread per selected node");
+constexpr int kMaskWords = kMaxLayer / 32;
 
 __device__ __forceinline__ uint64_t score_key(double s) {
   uint64_t u = static_cast<uint64_t>(__double_as_longlong(s + 0.0));
@@ -35,247 +34,173 @@ __device__ __forceinline__ double key_score(uint64_t k) {
   return __longlong_as_double(static_cast<long long>(u));
 }
 
-__device__ __forceinline__ Item shfl_item(const Item& a, int src) {
-  Item o;
-  o.key = __shfl_sync(kFull, a.key, src);
-  o.aux = __shfl_sync(kFull, a.aux, src);
-  return o;
-}
-
-// One compare-exchange layer of a bitonic network over the blocked layout i = lane*kE + e.
-// `desc_mask`: element i sorts descending iff (i & desc_mask) == 0 (0 = all descending).
-template <int STRIDE>
-__device__ __forceinline__ void bitonic_layer(Item (&x)[kE], int lane, int desc_mask) {
-  if constexpr (STRIDE < kE) {
-#pragma unroll
-    for (int e = 0; e < kE; ++e) {
-      if ((e & STRIDE) == 0) {
-        int i = lane * kE + e;
-        bool desc = (i & desc_mask) == 0;
-        Item a = x[e], b = x[e | STRIDE];
-        bool a_first = better(a, b);
-        bool keep = (a_first == desc);
-        x[e] = keep ? a : b;
-        x[e | STRIDE] = keep ? b : a;
-      }
-    }
-  } else {
-    constexpr int LS = STRIDE / kE;
-    bool lower = (lane & LS) == 0;
-#pragma unroll
-    for (int e = 0; e < kE; ++e) {
-      int i = lane * kE + e;
-      bool desc = (i & desc_mask) == 0;
-      Item o = shfl_item(x[e], lane ^ LS);
-      bool mine_better = better(x[e], o);
-      bool take_better = (lower == desc);
-      x[e] = (mine_better == take_better) ? x[e] : o;
-    }
-  }
-}
-
-template <int SIZE>
-__device__ __forceinline__ void bitonic_merge_from(Item (&x)[kE], int lane, int desc_mask) {
-  if constexpr (SIZE >= 2) {
-    bitonic_layer<SIZE / 2>(x, lane, desc_mask);
-    bitonic_merge_from<SIZE / 2>(x, lane, desc_mask);
-  }
-}
-
-template <int SIZE>
-__device__ __forceinline__ void bitonic_sort_upto(Item (&x)[kE], int lane) {
-  if constexpr (SIZE >= 2) {
-    bitonic_sort_upto<SIZE / 2>(x, lane);
-    bitonic_merge_from<SIZE>(x, lane, SIZE == kN ? 0 : SIZE);
-  }
-}
-
-// Full descending sort of the 128 items held by the warp.
-__device__ __forceinline__ void warp_sort_desc(Item (&x)[kE], int lane) {
-  bitonic_sort_upto<kN>(x, lane);
-}
-
-// a, b sorted descending -> a = the 128 best of the union, sorted descending.
-__device__ __forceinline__ void warp_merge_top(Item (&a)[kE], const Item (&b)[kE], int lane) {
-#pragma unroll
-  for (int e = 0; e < kE; ++e) {
-    Item o = shfl_item(b[kE - 1 - e], 31 - lane);  // b reversed
-    if (better(o, a[e])) a[e] = o;
-  }
-  bitonic_merge_from<kN>(a, lane, 0);
-}
-
-struct WarpSmem {
-  int fpool[kMaxDepth][16];  // fpool[d][j]: pool index of frontier slot j at depth d (1..D-1)
-  double fcum[16];           // cumulative score of the current frontier
-  double score[kN];
-  int sel_pool[kN];
-  int parent[kN];
+struct TreeSmem {
+  uint64_t ukey[kMaxLayer];             // keys of the layer in work, by candidate index q
+  double fcum[2][kMaxTopK];             // cumulative score of the frontier (double-buffered)
+  int fpool[kMaxDepth][kMaxTopK];       // fpool[d][j]: pool index of frontier slot j at depth d
+  unsigned selmask[kMaxDepth][kMaskWords];  // selected candidates of each layer, bit q
+  int sel_before[kMaxDepth + 1];        // selected nodes in the layers before this one
+  int parent[kMaxNodes];
 };
 
-__global__ void __launch_bounds__(kWarpsPerCta * 32) tree_build_kernel(TreeBuildArgs a) {
-  __shared__ WarpSmem smem[kWarpsPerCta];
-  const int lane = threadIdx.x & 31;
-  const int wic = threadIdx.x >> 5;
-  const int tree = blockIdx.x * kWarpsPerCta + wic;
-  if (tree >= a.n_trees) return;
-  WarpSmem& sm = smem[wic];
+// Entries of a descending list that come before x; equal keys come before x iff `ties_first`.
+__device__ __forceinline__ int count_ahead(const uint64_t* list, int n, uint64_t x,
+                                           bool ties_first) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    const uint64_t y = list[mid];
+    if (y > x || (y == x && ties_first)) lo = mid + 1; else hi = mid;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ int bits_below(const unsigned (&m)[kMaskWords], int q) {
+  int n = 0;
+#pragma unroll
+  for (int w = 0; w < kMaskWords; ++w) {
+    if (w < (q >> 5)) n += __popc(m[w]);
+    else if (w == (q >> 5)) n += __popc(m[w] & ((1u << (q & 31)) - 1u));
+  }
+  return n;
+}
+
+__global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs a) {
+  extern __shared__ __align__(16) unsigned char dyn[];
+  __shared__ TreeSmem sm;
+  const int tid = threadIdx.x;
+  const int tree = blockIdx.x;
   const int D = a.D, k = a.k, g = a.g, R = a.R, kk = a.k * a.k;
+  const int P = k + (D - 1) * kk;
+  uint64_t* skey = reinterpret_cast<uint64_t*>(dyn);       // [P] every layer, sorted
+  uint8_t* sq = reinterpret_cast<uint8_t*>(skey + P);      // [P] candidate index at that rank
   const double* lse = a.row_lse + static_cast<size_t>(tree) * R;
   const int32_t* top_id = a.top_id + static_cast<size_t>(tree) * R * k;
   const float* top_z = a.top_z + static_cast<size_t>(tree) * R * k;
+  auto list_off = [&](int l) { return l == 0 ? 0 : k + (l - 1) * kk; };  // = pool index base
+  auto list_len = [&](int l) { return l == 0 ? k : kk; };
 
+  if (tid < D * kMaskWords) (&sm.selmask[0][0])[tid] = 0;
   // ---- depth 1: the root's k best tokens, already in rank order = pool order
-  Item best[kE];  // running global ranking (score desc, pool index asc)
-  {
-    const double l0 = lse[0];
-#pragma unroll
-    for (int e = 0; e < kE; ++e) {
-      int c = lane * kE + e;
-      if (c < k) {
-        double sc = static_cast<double>(top_z[c]) - l0;
-        best[e].key = score_key(sc);
-        best[e].aux = c;
-        if (D > 1) {
-          sm.fcum[c] = sc;
-          sm.fpool[1][c] = c;
-        }
-      } else {
-        best[e].key = 0;
-        best[e].aux = kInvalidAux;
-      }
+  if (tid < k) {
+    const double sc = static_cast<double>(top_z[tid]) - lse[0];
+    skey[tid] = score_key(sc);
+    sq[tid] = static_cast<uint8_t>(tid);
+    if (D > 1) {
+      sm.fcum[0][tid] = sc;
+      sm.fpool[1][tid] = tid;
     }
   }
-  __syncwarp();
+  __syncthreads();
 
-  // ---- depths 2..D: k*k candidates per layer
+  // ---- depths 2..D: k*k candidates per layer, rank = position in (score desc, q asc) order
+  int cur = 0;
   for (int d = 2; d <= D; ++d) {
-    const int base = k + (d - 2) * kk;
-    Item cand[kE];
-#pragma unroll
-    for (int e = 0; e < kE; ++e) {
-      int q = lane * kE + e;
-      if (q < kk) {
-        int j = q / k, c = q - j * k;
-        int row = 1 + (d - 2) * k + j;
-        double sc = sm.fcum[j] + (static_cast<double>(top_z[row * k + c]) - lse[row]);
-        cand[e].key = score_key(sc);
-        cand[e].aux = base + q;
-      } else {
-        cand[e].key = 0;
-        cand[e].aux = kInvalidAux;
+    const int base = list_off(d - 1);
+    const int j = tid / k, c = tid - j * k;
+    double sc = 0.0;
+    uint64_t key = 0;
+    if (tid < kk) {
+      const int row = 1 + (d - 2) * k + j;
+      sc = sm.fcum[cur][j] + (static_cast<double>(top_z[row * k + c]) - lse[row]);
+      key = score_key(sc);
+      sm.ukey[tid] = key;
+    }
+    __syncthreads();
+    if (tid < kk) {
+      int rank = c;  // the children of one parent are in order already
+      for (int jp = 0; jp < k; ++jp)
+        if (jp != j) rank += count_ahead(&sm.ukey[jp * k], k, key, jp < j);
+      skey[base + rank] = key;
+      sq[base + rank] = static_cast<uint8_t>(tid);
+      if (d < D && rank < k) {
+        sm.fcum[cur ^ 1][rank] = sc;
+        sm.fpool[d][rank] = base + tid;
       }
     }
-    __syncwarp();  // all lanes have read fcum
-    warp_sort_desc(cand, lane);
-    if (d < D) {
-#pragma unroll
-      for (int e = 0; e < kE; ++e) {
-        int rank = lane * kE + e;
-        if (rank < k) {
-          sm.fcum[rank] = key_score(cand[e].key);
-          sm.fpool[d][rank] = static_cast<int>(cand[e].aux);
-        }
-      }
-    }
-    warp_merge_top(best, cand, lane);
-    __syncwarp();
+    __syncthreads();
+    cur ^= 1;
   }
 
-  // ---- the g best, re-listed in ascending pool index
-#pragma unroll
-  for (int e = 0; e < kE; ++e) {
-    int i = lane * kE + e;
-    sm.score[i] = key_score(best[e].key);
-    Item it;
-    if (i < g) {
-      it.key = ~static_cast<uint64_t>(best[e].aux);  // smaller pool index = larger key
-      it.aux = i;
-    } else {
-      it.key = 0;
-      it.aux = kInvalidAux;
+  // ---- global top-g: rank among all candidates = rank in the layer + entries ahead in
+  //      every other layer.  Items are (layer l, rank r < min(len, g)), dealt round-robin.
+  int n_items = 0;
+  for (int l = 0; l < D; ++l) n_items += min(list_len(l), g);
+  auto item = [&](int t, int& l, int& r) {
+    l = 0;
+    int n = min(list_len(0), g);
+    while (t >= n) {
+      t -= n;
+      ++l;
+      n = min(list_len(l), g);
     }
-    best[e] = it;
-  }
-  __syncwarp();
-  warp_sort_desc(best, lane);
-  double node_score[kE];
-  int node_pool[kE];
-#pragma unroll
-  for (int e = 0; e < kE; ++e) {
-    int n = lane * kE + e;
-    if (n < g) {
-      node_pool[e] = static_cast<int>(~best[e].key);
-      node_score[e] = sm.score[best[e].aux];
-      sm.sel_pool[n] = node_pool[e];
-    } else {
-      node_pool[e] = -1;
-      node_score[e] = 0.0;
+    r = t;
+  };
+  for (int t = tid; t < n_items; t += kTreeThreads) {
+    int l, r;
+    item(t, l, r);
+    const uint64_t x = skey[list_off(l) + r];
+    int rank = r;
+    for (int lp = 0; lp < D && rank < g; ++lp)
+      if (lp != l) rank += count_ahead(skey + list_off(lp), list_len(lp), x, lp < l);
+    if (rank < g) {
+      const int q = sq[list_off(l) + r];
+      atomicOr(&sm.selmask[l][q >> 5], 1u << (q & 31));
     }
   }
-  __syncwarp();
+  __syncthreads();
+  if (tid <= D) {
+    int n = 0;
+    for (int l = 0; l < tid; ++l)
+#pragma unroll
+      for (int w = 0; w < kMaskWords; ++w) n += __popc(sm.selmask[l][w]);
+    sm.sel_before[tid] = n;
+  }
+  __syncthreads();
 
-  // ---- per-node fields
+  // ---- per-node fields, listed in ascending pool index
   const size_t obase = static_cast<size_t>(tree) * g;
-#pragma unroll
-  for (int e = 0; e < kE; ++e) {
-    int n = lane * kE + e;
-    if (n < g) {
-      int p = node_pool[e];
-      int depth, c, ctx, par = -1;
-      if (p < k) {
-        depth = 1;
-        c = p;
-        ctx = 0;
-      } else {
-        int dd = (p - k) / kk;
-        int q = (p - k) - dd * kk;
-        int j = q / k;
-        depth = dd + 2;
-        c = q - j * k;
-        ctx = 1 + dd * k + j;
-        int pp = sm.fpool[depth - 1][j];
-        int lo = 0, hi = g - 1;  // the parent is selected whenever the child is
-        while (lo < hi) {
-          int mid = (lo + hi) >> 1;
-          if (sm.sel_pool[mid] < pp) lo = mid + 1; else hi = mid;
-        }
-        par = lo;
-      }
-      int slot = -1;
-      if (depth < D) {
-        for (int j = 0; j < k; ++j)
-          if (sm.fpool[depth][j] == p) slot = j;
-      }
-      sm.parent[n] = par;
-      a.out.node_token[obase + n] = top_id[ctx * k + c];
-      a.out.node_parent[obase + n] = par;
-      a.out.node_depth[obase + n] = depth;
-      a.out.node_ctx_row[obase + n] = ctx;
-      a.out.node_slot[obase + n] = slot;
-      a.out.node_pool[obase + n] = p;
-      a.out.node_logp[obase + n] =
-          static_cast<float>(static_cast<double>(top_z[ctx * k + c]) - lse[ctx]);
-      a.out.node_score[obase + n] = node_score[e];
+  for (int t = tid; t < n_items; t += kTreeThreads) {
+    int l, r;
+    item(t, l, r);
+    const int off = list_off(l);
+    const int q = sq[off + r];
+    if (!((sm.selmask[l][q >> 5] >> (q & 31)) & 1u)) continue;
+    const int n = sm.sel_before[l] + bits_below(sm.selmask[l], q);
+    const int depth = l + 1;
+    int c = q, ctx = 0, par = -1;
+    if (l > 0) {
+      const int j = q / k;
+      c = q - j * k;
+      ctx = 1 + (l - 1) * k + j;
+      // the parent scores at least as high and has the lower pool index: it is selected too
+      const int qp = sm.fpool[l][j] - list_off(l - 1);
+      par = sm.sel_before[l - 1] + bits_below(sm.selmask[l - 1], qp);
     }
+    sm.parent[n] = par;
+    a.out.node_token[obase + n] = top_id[ctx * k + c];
+    a.out.node_parent[obase + n] = par;
+    a.out.node_depth[obase + n] = depth;
+    a.out.node_ctx_row[obase + n] = ctx;
+    a.out.node_slot[obase + n] = (depth < D && r < k) ? r : -1;  // frontier slot = layer rank
+    a.out.node_pool[obase + n] = off + q;
+    a.out.node_logp[obase + n] =
+        static_cast<float>(static_cast<double>(top_z[ctx * k + c]) - lse[ctx]);
+    a.out.node_score[obase + n] = key_score(skey[off + r]);
   }
-  __syncwarp();
+  __syncthreads();
 
   // ---- ancestor mask: bit a of row n set iff a is n or an ancestor of n
   const int W = (g + 63) / 64;
-#pragma unroll
-  for (int e = 0; e < kE; ++e) {
-    int n = lane * kE + e;
-    if (n < g) {
-      uint64_t w0 = 0, w1 = 0;
-      int x = n;
-      for (int step = 0; step <= D && x >= 0; ++step) {
-        if (x < 64) w0 |= 1ull << x; else w1 |= 1ull << (x - 64);
-        x = sm.parent[x];
-      }
-      a.out.node_mask[(obase + n) * W] = w0;
-      if (W > 1) a.out.node_mask[(obase + n) * W + 1] = w1;
+  if (tid < g) {
+    uint64_t w0 = 0, w1 = 0;
+    int x = tid;
+    for (int step = 0; step <= D && x >= 0; ++step) {
+      if (x < 64) w0 |= 1ull << x; else w1 |= 1ull << (x - 64);
+      x = sm.parent[x];
     }
+    a.out.node_mask[(obase + tid) * W] = w0;
+    if (W > 1) a.out.node_mask[(obase + tid) * W + 1] = w1;
   }
 }
 
@@ -283,8 +208,9 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_build_kernel(TreeBuild
 
 cudaError_t launch_tree_build(const TreeBuildArgs& a, cudaStream_t stream, int64_t* launches) {
   if (a.n_trees <= 0) return cudaSuccess;
-  dim3 grid((a.n_trees + kWarpsPerCta - 1) / kWarpsPerCta), block(kWarpsPerCta * 32);
-  tree_build_kernel<<<grid, block, 0, stream>>>(a);
+  const int P = a.k + (a.D - 1) * a.k * a.k;
+  const size_t dyn = static_cast<size_t>(P) * (sizeof(uint64_t) + 1);
+  tree_build_kernel<<<a.n_trees, kTreeThreads, dyn, stream>>>(a);
   ++*launches;
   return cudaGetLastError();
 }

@@ -69,6 +69,26 @@ def test_variants_max_mean_unbiased_nodebias(harness):
     harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(unbiased=True, debias=False))
 
 
+def test_grad_live_rows_flag_leaves_the_other_rows_untouched(harness):
+    from paper_2509_22134_b200 import binding as gto
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.WORKLOADS[1].with_B(32)
+    p_ref, data = harness.run_pass(w, DEV)
+    p = GtoPass(w, DEV, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS)
+    p.build_tree(data["draft"])
+    p.tree_reward(data["target"], data["d2t"])
+    p.set_old_logp_from_path()
+    p.grad.fill_(7.0)
+    p.surrogate_grad(data["draft"])
+    torch.cuda.synchronize()
+    j = torch.arange(w.D, device=DEV)[None, :]
+    live = (j < p.reward["path_len"][:, None]) & (p.stats["coeff"][:, None] != 0)
+    assert int(live.sum()) > 0
+    assert torch.equal(p.grad[live], p_ref.grad[live])
+    assert bool((p.grad[~live] == 7.0).all())
+    assert bool((p_ref.grad[~live] == 0.0).all())
+
+
 def test_deterministic_integer_outputs(harness):
     w = synth.WORKLOADS[1].with_B(32)
     p1, data = harness.run_pass(w, DEV)
