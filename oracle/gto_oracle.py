@@ -17,6 +17,7 @@ Steps and the passages they follow:
   group_advantages      Sec. 3.2 Eq. 9-10 (debias, standardise)
   clipped_surrogate     Sec. 3.2 Eq. 11-12 (length-normalised ratio, PPO clip)
   surrogate_grad_rows   derivative of Eq. 12 with respect to the draft logits
+  token_loss            Sec. 3.2 Eq. 13 and App. B: teacher-to-student cross-entropy per prefix
 
 Readings fixed where the paper is silent (all listed in the design notes):
   * global acceptance score = sum of draft log-probabilities along the path;
@@ -27,7 +28,9 @@ Readings fixed where the paper is silent (all listed in the design notes):
   * the sequences S_i of Eq. 2 are the root-to-leaf paths of the selected tree;
   * "accepted" means greedy (temperature 0) verification; the bonus token is not counted;
   * std is the population std; groups are consecutive blocks of m positions;
-  * advantages and the old-policy log-probabilities are constants for the gradient.
+  * advantages and the old-policy log-probabilities are constants for the gradient;
+  * with a reduced draft vocabulary the target distribution of the token-level loss is
+    renormalised over the mapped ids.
 
 Pins (tests/test_oracle_*.py): naive long-double log-sum-exp, brute-force sort,
 an independent path-enumerating tree builder, special cases k=1 / D=1 / g=P, the
@@ -413,3 +416,28 @@ def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, ag
         grad[i] = surrogate_grad_rows(rows, lse, list(path_tok[i, :l]), sur["coeff"][i], D, V)
     return dict(fwd=fwd, R=R, A=A, path_len=path_len, path_logp=path_logp, path_row=path_row,
                 path_token=path_tok, old=old, sur=sur, grad=grad)
+
+
+# ------------------------------------------------------------------ token-level loss
+def token_loss(z_draft, z_target, d2t=None):
+    """Token-level loss of Eq. 13 / App. B for one teacher-forced prefix: the cross-entropy
+    H(p_T, p_M) = -sum_v p_T(v) log p_M(v) from the target's next-token distribution to the
+    draft's, and its derivative with respect to the draft logits, p_M - p_T.
+
+    z_draft: [V_d] draft logits of the prefix; z_target: [V_t] target logits of the same
+    prefix.  With a reduced draft vocabulary (d2t: draft id -> target id) the target
+    distribution is the softmax of the target logits at the mapped ids only, so that both
+    distributions live on the draft vocabulary (the paper sums over one common vocabulary).
+    Returns (H, grad[V_d]).
+    """
+    zd = np.asarray(z_draft, dtype=np.float64)
+    zt = np.asarray(z_target, dtype=np.float64)
+    if d2t is not None:
+        zt = zt[np.asarray(d2t, dtype=np.int64)]
+    assert zd.shape == zt.shape
+    md, mt = np.max(zd), np.max(zt)
+    log_pm = zd - (md + np.log(np.sum(np.exp(zd - md))))
+    log_pt = zt - (mt + np.log(np.sum(np.exp(zt - mt))))
+    p_t = np.exp(log_pt)
+    H = -float(np.sum(p_t * log_pm))
+    return H, np.exp(log_pm) - p_t
