@@ -282,6 +282,23 @@ def run_gpu(args, w, rank, world, local_rank):
     launches = p.launches() - launches0
     assert p.status() == 0
 
+    # ---- next-row kernel, timed on its own (not part of the step): token-level loss
+    extras = {}
+    if not args.no_e2e:
+        gto.gto_kernel_timing(p.ctx, True)
+        for _ in range(3):
+            p.token_loss(data["draft"], data["target"], data["d2t"], 1.0 / w.B)
+        gto.gto_kernel_times(p.ctx)
+        for _ in range(args.steps):
+            p.token_loss(data["draft"], data["target"], data["d2t"], 1.0 / w.B)
+        tot, cnt = gto.gto_kernel_times(p.ctx)["token_loss"]
+        gto.gto_kernel_timing(p.ctx, False)
+        tok_bytes = w.B * 3 * w.V_draft * w.elem_bytes   # draft row, mapped target logits, gradient row
+        extras["token_loss"] = {"ms": tot / cnt, "algorithmic_bytes": tok_bytes,
+                                "gbs": tok_bytes / (tot / cnt * 1e-3) / 1e9,
+                                "note": "Eq. 13 on the B root rows; the id-map gather touches "
+                                        "nearly every 32-byte sector of the target row"}
+
     # ---- end to end: host buffers, copies inside the timed region
     e2e = run_e2e(args, w, dev, b0, world) if not args.no_e2e else None
     if e2e is None:
@@ -329,7 +346,8 @@ def run_gpu(args, w, rank, world, local_rank):
                     "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                     "positions_per_step": e2e["positions_per_step"], "steps": e2e["steps"]},
             "gpu_launches": launches,
-            "roofline": roofline}
+            "roofline": roofline,
+            "extras": extras}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, dev)
     print(json.dumps(line), flush=True)

@@ -178,6 +178,25 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft_logits,
                                     const float* old_logp, void* grad,
                                     const gto_grad_stats* out, void* stream);
 
+/* Token-level loss of Eq. 13 / App. B. */
+typedef struct {
+  double* loss;   /* [B] H(p_T, p_M) of the position's prefix                              */
+  double* lse_t;  /* [B] log-sum-exp of the target logits over the (mapped) draft vocabulary */
+} gto_token_stats;
+
+/* Token-level loss L_token of Eq. 13 (defined in App. B): for every position b the
+ * cross-entropy H(p_T, p_M) = -sum_v p_T(v) log p_M(v) from the target's next-token
+ * distribution to the draft's under the same teacher-forced prefix, i.e. on the root context
+ * rows draft[0,b,0,0,:] and target[0,b,0,:].  With a reduced draft vocabulary p_T is the
+ * softmax of the target logits at the mapped ids d2t[0..V_draft) (NULL = identity).  Writes
+ * out->loss[b] and grad_root[b,:] = weight * (p_M - p_T), the derivative of weight * H with
+ * respect to the draft logits of that row ([B, V_draft], logit dtype, every entry written);
+ * a trainer passes weight = 1 / (number of supervised positions).  Needs tree->row_lse from
+ * gto_build_tree on the same draft logits. */
+gto_status gto_token_loss(gto_ctx* ctx, const void* draft_logits, const void* target_logits,
+                          const int32_t* d2t, const gto_tree* tree, float weight,
+                          void* grad_root, const gto_token_stats* out, void* stream);
+
 /* Synchronises `stream`, then reads and clears the device status word:
  * *host_code = GTO_OK, GTO_ERR_NONFINITE or GTO_ERR_TIMEOUT. */
 gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code);
@@ -194,7 +213,8 @@ enum {
   GTO_K_TREE_REWARD = 4, /* Eq. 3-5 and the longest accepted sequence                      */
   GTO_K_GROUP_STATS = 5, /* Eq. 9-12 per group                                             */
   GTO_K_GRAD_ROWS = 6,   /* derivative of Eq. 12 into the draft rows of the accepted path  */
-  GTO_K_COUNT = 7
+  GTO_K_TOKEN_LOSS = 7,  /* Eq. 13 / App. B: cross-entropy and its gradient on the root rows */
+  GTO_K_COUNT = 8
 };
 
 /* Per-kernel device timing, off by default.  While enabled, every launch is bracketed by

@@ -44,6 +44,7 @@ _REWARD_FIELDS = [("reward", torch.float64), ("etree", torch.float64), ("n_leave
                   ("row_argmax_t", torch.int32), ("path_len", torch.int32),
                   ("path_node", torch.int32), ("path_row", torch.int32),
                   ("path_token", torch.int32), ("path_logp", torch.float32)]
+_TOKEN_FIELDS = [("loss", torch.float64), ("lse_t", torch.float64)]
 _STATS_FIELDS = [("R", torch.float64), ("adv", torch.float64), ("ratio", torch.float64),
                  ("coeff", torch.float64), ("active", torch.int32), ("loss", torch.float64)]
 
@@ -55,6 +56,7 @@ def _struct(name, fields):
 gto_tree = _struct("gto_tree", _TREE_FIELDS)
 gto_reward = _struct("gto_reward", _REWARD_FIELDS)
 gto_grad_stats = _struct("gto_grad_stats", _STATS_FIELDS)
+gto_token_stats = _struct("gto_token_stats", _TOKEN_FIELDS)
 
 _vp = ctypes.c_void_p
 _lib.gto_create.argtypes = [ctypes.POINTER(_vp), ctypes.POINTER(gto_config), ctypes.c_int]
@@ -66,6 +68,9 @@ _lib.gto_build_tree_noalloc.restype = ctypes.c_int
 _lib.gto_tree_reward.argtypes = [_vp, ctypes.POINTER(gto_tree), _vp, _vp, ctypes.POINTER(gto_reward), _vp]
 _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ctypes.POINTER(gto_reward),
                                           _vp, _vp, ctypes.POINTER(gto_grad_stats), _vp]
+_lib.gto_token_loss.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(gto_tree), ctypes.c_float, _vp,
+                                ctypes.POINTER(gto_token_stats), _vp]
+_lib.gto_token_loss.restype = ctypes.c_int
 _lib.gto_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_int32)]
 _lib.gto_launch_count.argtypes = [_vp]
 _lib.gto_launch_count.restype = ctypes.c_int64
@@ -189,6 +194,24 @@ def gto_group_surrogate_grad(ctx: int, draft: torch.Tensor, tree: dict, reward: 
                                          _stream_ptr(stream)), "gto_group_surrogate_grad")
 
 
+def alloc_token_stats(cfg: gto_config, device) -> dict:
+    return {n: torch.empty((cfg.B,), dtype=dt, device=device) for n, dt in _TOKEN_FIELDS}
+
+
+def gto_token_loss(ctx: int, draft: torch.Tensor, target: torch.Tensor, d2t, tree: dict, weight: float,
+                   grad_root: torch.Tensor, stats: dict, stream=None):
+    assert draft.is_cuda and draft.is_contiguous() and target.is_cuda and target.is_contiguous()
+    assert grad_root.is_cuda and grad_root.is_contiguous() and grad_root.dtype == draft.dtype
+    if d2t is not None:
+        assert d2t.is_cuda and d2t.dtype == torch.int32 and d2t.is_contiguous()
+    t = _fill(gto_tree, _TREE_FIELDS, tree)
+    s = _fill(gto_token_stats, _TOKEN_FIELDS, stats)
+    _check(_lib.gto_token_loss(ctx, draft.data_ptr(), target.data_ptr(),
+                               None if d2t is None else d2t.data_ptr(), ctypes.byref(t),
+                               ctypes.c_float(weight), grad_root.data_ptr(), ctypes.byref(s),
+                               _stream_ptr(stream)), "gto_token_loss")
+
+
 def gto_device_status(ctx: int, stream=None) -> int:
     code = ctypes.c_int32(0)
     _check(_lib.gto_device_status(ctx, _stream_ptr(stream), ctypes.byref(code)), "gto_device_status")
@@ -200,7 +223,7 @@ def gto_launch_count(ctx: int) -> int:
 
 
 KERNEL_NAMES = ["draft_rows", "tree_build", "reward_plan", "target_rows", "tree_reward",
-                "group_stats", "grad_rows"]   # GTO_K_* order
+                "group_stats", "grad_rows", "token_loss"]   # GTO_K_* order
 
 
 def gto_kernel_timing(ctx: int, enable: bool):
@@ -218,4 +241,4 @@ def gto_kernel_times(ctx: int, stream=None) -> dict:
 
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
            "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
-           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc"]
+           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss"]

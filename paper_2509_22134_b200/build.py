@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libgto.so")
 SOURCES = ["gto_api.cu", "row_reduce.cu", "tree_build.cu", "tree_reward.cu", "surrogate_grad.cu",
-           "build_tree_noalloc.cu"]
+           "build_tree_noalloc.cu", "token_loss.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

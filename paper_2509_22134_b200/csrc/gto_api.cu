@@ -289,6 +289,34 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
   return GTO_OK;
 }
 
+gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, const int32_t* d2t,
+                          const gto_tree* tree, float weight, void* grad_root,
+                          const gto_token_stats* out, void* stream) {
+  if (!ctx || !draft || !target || !tree || !grad_root || !out || !aligned16(draft) ||
+      !aligned16(target) || !aligned16(grad_root) || !all_set(tree) || !all_set(out))
+    return GTO_ERR_INVALID_ARG;
+  const gto_config& c = ctx->cfg;
+  if (!d2t && c.V_draft != c.V_target) return GTO_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  if (!guard.ok) return GTO_ERR_CUDA;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  gto::TokenLossArgs a{};
+  a.B = c.B; a.k = c.k; a.R = ctx->R; a.V_draft = c.V_draft; a.V_target = c.V_target;
+  a.dtype = c.logit_dtype;
+  a.weight = weight;
+  a.draft = draft;
+  a.target = target;
+  a.d2t = d2t;
+  a.row_lse = tree->row_lse;
+  a.grad_root = grad_root;
+  a.loss = out->loss;
+  a.lse_t = out->lse_t;
+  a.status = ctx->status;
+  LaunchSpan span(ctx, GTO_K_TOKEN_LOSS, s);
+  if (gto::launch_token_loss(a, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  return GTO_OK;
+}
+
 gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code) {
   if (!ctx || !host_code) return GTO_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);

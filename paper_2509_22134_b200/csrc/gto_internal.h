@@ -71,6 +71,20 @@ struct GradArgs {
   void* grad;
   gto_grad_stats out;
 };
+struct TokenLossArgs {
+  int B, k, R, V_draft, V_target, dtype;
+  float weight;
+  const void* draft;       // [G,B,D,k,V_draft]; row [0,b,0,0,:] is read
+  const void* target;      // [G,B,R,V_target]; row [0,b,0,:] is read
+  const int32_t* d2t;      // [V_draft] or null (identity)
+  const double* row_lse;   // [G*B*R] draft log-sum-exp (entry of row 0 of tree (0,b))
+  void* grad_root;         // [B, V_draft] in the logit dtype
+  double* loss;            // [B]
+  double* lse_t;           // [B]
+  int32_t* status;
+};
+cudaError_t launch_token_loss(const TokenLossArgs& a, cudaStream_t stream, int64_t* launches);
+
 cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches);
 

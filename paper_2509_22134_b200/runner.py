@@ -63,6 +63,15 @@ class GtoPass:
         self.tree_reward(target, d2t, stream)
         self.surrogate_grad(draft, stream)
 
+    def token_loss(self, draft, target, d2t, weight: float = 1.0, stream=None):
+        """Token-level loss on the root rows; allocates its outputs on first use."""
+        if not hasattr(self, "token_stats"):
+            self.token_stats = gto.alloc_token_stats(self.cfg, self.device)
+            self.grad_root = torch.empty((self.w.B, self.w.V_draft), dtype=self.w.torch_dtype,
+                                         device=self.device)
+        gto.gto_token_loss(self.ctx, draft, target, d2t, self.tree, weight, self.grad_root,
+                           self.token_stats, stream)
+
     def status(self) -> int:
         return gto.gto_device_status(self.ctx)
 

@@ -89,6 +89,37 @@ def test_grad_live_rows_flag_leaves_the_other_rows_untouched(harness):
     assert bool((p_ref.grad[~live] == 0.0).all())
 
 
+@pytest.mark.parametrize("kw", [
+    dict(B=16, V_draft=4104, V_target=4104, D=3, k=4, g=12, dtype="bf16", seed=21),
+    dict(B=16, V_draft=2048, V_target=8200, D=3, k=4, g=12, dtype="bf16", seed=22),   # id map
+    dict(B=8, V_draft=1000, V_target=1000, D=2, k=4, g=8, dtype="f32", seed=23),
+    dict(B=8, V_draft=32000, V_target=128256, D=2, k=10, g=20, dtype="bf16", seed=24),
+])
+def test_token_loss_matches_the_oracle(harness, kw):
+    """Eq. 13 / App. B on the root rows: loss 1e-4 relative; gradient entries are
+    weight * (p_M - p_T) in [-weight, weight], stored in the logit dtype, so bf16 rounding
+    alone is up to 2^-9 relative: tolerance 2e-3 * weight absolute + 2^-8 relative."""
+    from oracle import gto_oracle as orc
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.Workload("tok", **kw)
+    data = synth.generate(w, DEV)
+    p = GtoPass(w, DEV)
+    p.build_tree(data["draft"])
+    weight = 0.5
+    p.token_loss(data["draft"], data["target"], data["d2t"], weight)
+    assert p.status() == 0
+    loss = p.token_stats["loss"].cpu().numpy()
+    grad = p.grad_root.float().cpu().numpy().astype(np.float64)
+    d2t = None if data["d2t"] is None else data["d2t"].cpu().numpy()
+    zd = data["draft"][0, :, 0, 0].float().cpu().numpy()
+    zt = data["target"][0, :, 0].float().cpu().numpy()
+    for b in range(w.B):
+        H, g = orc.token_loss(zd[b], zt[b], d2t)
+        assert abs(loss[b] - H) <= 1e-4 * max(1.0, abs(H)), (b, loss[b], H)
+        err = np.abs(grad[b] - weight * g)
+        assert np.all(err <= 2e-3 * weight + 2.0 ** -8 * np.abs(weight * g)), (b, err.max())
+
+
 def test_deterministic_integer_outputs(harness):
     w = synth.WORKLOADS[1].with_B(32)
     p1, data = harness.run_pass(w, DEV)
