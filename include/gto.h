@@ -52,6 +52,8 @@ typedef enum { GTO_AGG_LSE = 0, GTO_AGG_MAX = 1, GTO_AGG_MEAN = 2 } gto_agg;
 enum {
   GTO_FLAG_STD_UNBIASED = 1u, /* Eq. 10 with the sample std (divide by m-1)             */
   GTO_FLAG_NO_DEBIAS = 2u,    /* Eq. 9 switched off: R_i = r(T_i) (debiasing ablation)  */
+  GTO_FLAG_SEQ_ALL_NODES = 8u, /* Eq. 5 over the root-to-node sequence of every selected node
+                                  instead of the root-to-leaf sequences only                 */
   GTO_FLAG_GRAD_LIVE_ROWS = 4u /* gto_group_surrogate_grad writes only the rows that carry a
                                   gradient (j < path_len[b] and coeff[b] != 0) and leaves the
                                   rest of grad untouched, instead of filling it with zeros   */
@@ -196,6 +198,14 @@ typedef struct {
 gto_status gto_token_loss(gto_ctx* ctx, const void* draft_logits, const void* target_logits,
                           const int32_t* d2t, const gto_tree* tree, float weight,
                           void* grad_root, const gto_token_stats* out, void* stream);
+
+/* SampleGroups of Algorithm 1 under Eq. 6-7: K non-overlapping groups of m adjacent positions
+ * of a sequence of length s; start indices are 1-based, 1 <= t_k <= s - m + 1 and
+ * t_{k+1} >= t_k + m.  Host-only (no device work): `u` is a HOST array of K uniforms in
+ * [0, 1) supplied by the caller, `starts` a HOST array that receives t_1 < ... < t_K.  Every
+ * admissible placement is equally likely for independent uniforms.  Returns
+ * GTO_ERR_INVALID_ARG when K*m > s or an argument is out of range. */
+gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts);
 
 /* Synchronises `stream`, then reads and clears the device status word:
  * *host_code = GTO_OK, GTO_ERR_NONFINITE or GTO_ERR_TIMEOUT. */

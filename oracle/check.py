@@ -48,7 +48,7 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
     for i in range(n):
         d_i = np.asarray(draft[:, i], dtype=np.float64)
         t_i = np.asarray(target[:, i], dtype=np.float64)
-        f = orc.position_forward(d_i, t_i, D, k, g, d2t, cfg.eta, agg)
+        f = orc.position_forward(d_i, t_i, D, k, g, d2t, cfg.eta, agg, getattr(cfg, "all_nodes", False))
         fwd.append(f)
         for t in range(G):
             tr = f["trees"][t]

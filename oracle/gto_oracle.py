@@ -208,13 +208,15 @@ def target_node_probs(tree, target, d2t=None):
     return p, lse_t
 
 
-def tree_reward(tree, p, eta=1.0, agg=AGG_LSE):
+def tree_reward(tree, p, eta=1.0, agg=AGG_LSE, all_nodes=False):
     """Draft Tree Reward, Eq. 3-5.
 
     Pp_n = product of p along the root-to-n path (Eq. 4), Lc_n = sum of Pp over the
     path (Eq. 3 for the sequence ending at n).  The sequences S_i are the
     root-to-leaf paths (leaf = selected node without a selected child), and
     r = (1/eta) log sum_i exp(eta L_i) (Eq. 5), or the Max / Average of Sec. 4.2.
+    With all_nodes the sequences are the root-to-node paths of every selected node (the
+    other reading of "N candidate sequences of length l_i <= d").
     Returns dict(r, Pp, Lc, leaves, etree) with etree = sum_n Pp_n (the exact
     expected number of accepted tokens when the target samples at temperature 1).
     """
@@ -231,7 +233,7 @@ def tree_reward(tree, p, eta=1.0, agg=AGG_LSE):
             has_child[a] = True
             Pp[n] = p[n] * Pp[a]
             Lc[n] = Lc[a] + Pp[n]
-    leaves = np.flatnonzero(~has_child)
+    leaves = np.arange(g) if all_nodes else np.flatnonzero(~has_child)
     L = Lc[leaves]
     if agg == AGG_LSE:
         M = np.max(eta * L)
@@ -357,7 +359,7 @@ def surrogate_grad_rows(draft_rows, row_lse, tokens, coeff, D, V):
 
 
 # ------------------------------------------------------------------ whole passes
-def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE):
+def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE, all_nodes=False):
     """Trees, rewards and the longest accepted sequence of one position.
 
     draft_b: [G, D, k, V_d], target_b: [G, R, V_t] with G = 2 (0 = current draft,
@@ -368,7 +370,7 @@ def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE)
     for t in range(G):
         tree = build_tree(draft_b[t], D, k, g)
         p, lse_t = target_node_probs(tree, target_b[t], d2t)
-        rw = tree_reward(tree, p, eta, agg)
+        rw = tree_reward(tree, p, eta, agg, all_nodes)
         rw["p"] = p
         rw["row_lse_t"] = lse_t
         trees.append(tree)
@@ -379,7 +381,7 @@ def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE)
 
 
 def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, agg=AGG_LSE,
-               delta=1e-6, eps=0.2, grad_scale=1.0, unbiased=False, debias=True):
+               delta=1e-6, eps=0.2, grad_scale=1.0, unbiased=False, debias=True, all_nodes=False):
     """The whole pass of Algorithm 1's inner loop on ONE group of m positions: trees and
     rewards of both drafts, the longest accepted sequences, Eq. 9-12 and the gradient rows.
     Sequences the functions above; adds no arithmetic of its own.
@@ -391,7 +393,8 @@ def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, ag
     """
     V = draft_g.shape[-1]
     fwd = [position_forward(np.asarray(draft_g[:, i], dtype=np.float64),
-                            np.asarray(target_g[:, i], dtype=np.float64), D, k, g, d2t, eta, agg)
+                            np.asarray(target_g[:, i], dtype=np.float64), D, k, g, d2t, eta, agg,
+                            all_nodes)
            for i in range(m)]
     r_cur = np.array([f["rewards"][0]["r"] for f in fwd])
     r_ref = np.array([f["rewards"][1]["r"] for f in fwd])
@@ -441,3 +444,18 @@ def token_loss(z_draft, z_target, d2t=None):
     p_t = np.exp(log_pt)
     H = -float(np.sum(p_t * log_pm))
     return H, np.exp(log_pm) - p_t
+
+
+# ------------------------------------------------------------------ grouping
+def sample_groups(s, m, K, u):
+    """SampleGroups of Algorithm 1 under the constraints of Eq. 6-7: K non-overlapping
+    groups of m adjacent positions of a sequence of length s, start indices 1-based with
+    1 <= t_k <= s - m + 1 and t_{k+1} >= t_k + m.  The paper does not say how the starts
+    are drawn; here every admissible placement is equally likely: the K uniforms u in
+    [0, 1) are turned into integers in [0, s - K m], sorted, and the k-th (0-based) is
+    shifted by k m.  Returns the start indices t_1 < ... < t_K.
+    """
+    assert K >= 0 and m >= 1 and K * m <= s
+    free = s - K * m
+    gaps = sorted(min(int(np.floor(float(x) * (free + 1))), free) for x in u[:K])
+    return [1 + gp + i * m for i, gp in enumerate(gaps)]

@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libgto.so")
 GTO_OK = 0
 GTO_F32, GTO_BF16 = 0, 1
 GTO_AGG_LSE, GTO_AGG_MAX, GTO_AGG_MEAN = 0, 1, 2
-GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS, GTO_FLAG_GRAD_LIVE_ROWS = 1, 2, 4
+GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS, GTO_FLAG_GRAD_LIVE_ROWS, GTO_FLAG_SEQ_ALL_NODES = 1, 2, 4, 8
 
 if not os.path.exists(LIB_PATH):
     raise RuntimeError(
@@ -71,6 +71,9 @@ _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ct
 _lib.gto_token_loss.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(gto_tree), ctypes.c_float, _vp,
                                 ctypes.POINTER(gto_token_stats), _vp]
 _lib.gto_token_loss.restype = ctypes.c_int
+_lib.gto_sample_groups.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                   ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int32)]
+_lib.gto_sample_groups.restype = ctypes.c_int
 _lib.gto_device_status.argtypes = [_vp, _vp, ctypes.POINTER(ctypes.c_int32)]
 _lib.gto_launch_count.argtypes = [_vp]
 _lib.gto_launch_count.restype = ctypes.c_int64
@@ -212,6 +215,14 @@ def gto_token_loss(ctx: int, draft: torch.Tensor, target: torch.Tensor, d2t, tre
                                _stream_ptr(stream)), "gto_token_loss")
 
 
+def gto_sample_groups(s: int, m: int, K: int, u) -> list:
+    """Start indices (1-based) of K non-overlapping groups of m adjacent positions (host only)."""
+    uu = (ctypes.c_double * max(K, 1))(*[float(x) for x in list(u)[:K]])
+    out = (ctypes.c_int32 * max(K, 1))()
+    _check(_lib.gto_sample_groups(s, m, K, uu, out), "gto_sample_groups")
+    return [int(out[i]) for i in range(K)]
+
+
 def gto_device_status(ctx: int, stream=None) -> int:
     code = ctypes.c_int32(0)
     _check(_lib.gto_device_status(ctx, _stream_ptr(stream), ctypes.byref(code)), "gto_device_status")
@@ -241,4 +252,4 @@ def gto_kernel_times(ctx: int, stream=None) -> dict:
 
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
            "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
-           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss"]
+           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss", "gto_sample_groups"]

@@ -1,4 +1,6 @@
 // C ABI of the GTO draft-tree pass: argument validation, workspace, launch sequencing.
+#include <algorithm>
+#include <cmath>
 #include <new>
 #include <vector>
 
@@ -246,6 +248,7 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   w.V_target = c.V_target;
   w.dtype = c.logit_dtype;
   w.agg = c.reward_agg;
+  w.flags = c.flags;
   w.eta = c.eta;
   w.target = target;
   w.d2t = d2t;
@@ -314,6 +317,22 @@ gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, c
   a.status = ctx->status;
   LaunchSpan span(ctx, GTO_K_TOKEN_LOSS, s);
   if (gto::launch_token_loss(a, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  return GTO_OK;
+}
+
+gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts) {
+  if (s < 0 || m < 1 || K < 0 || static_cast<int64_t>(K) * m > s) return GTO_ERR_INVALID_ARG;
+  if (K > 0 && (!u || !starts)) return GTO_ERR_INVALID_ARG;
+  // choose K sorted offsets in [0, s - K m] (with repetition), then spread them by k m:
+  // a bijection between such multisets and the admissible start sets
+  const int64_t free_slots = static_cast<int64_t>(s) - static_cast<int64_t>(K) * m;
+  for (int32_t i = 0; i < K; ++i) {
+    if (!(u[i] >= 0.0 && u[i] < 1.0)) return GTO_ERR_INVALID_ARG;
+    int64_t gap = static_cast<int64_t>(std::floor(u[i] * static_cast<double>(free_slots + 1)));
+    starts[i] = static_cast<int32_t>(std::min(gap, free_slots));
+  }
+  std::sort(starts, starts + K);
+  for (int32_t i = 0; i < K; ++i) starts[i] += 1 + i * m;
   return GTO_OK;
 }
 

@@ -52,6 +52,7 @@ cudaError_t launch_reward_plan(const RewardPlanArgs& a, cudaStream_t stream, int
 
 struct RewardArgs {
   int B, G, D, k, g, R, V_target, dtype, agg;
+  uint32_t flags;
   float eta;
   const void* target;
   const int32_t* d2t;

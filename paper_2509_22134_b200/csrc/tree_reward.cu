@@ -112,11 +112,12 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_reward_kernel(RewardAr
   }
   // ---- Eq. 5 over the leaves
   const double eta = static_cast<double>(a.eta);
+  const bool all_nodes = (a.flags & GTO_FLAG_SEQ_ALL_NODES) != 0;  // every node ends a sequence
   double mx = -INFINITY, sumL = 0.0, sumPp = 0.0;
   int leaves = 0;
   for (int n = lane; n < g; n += 32) {
     sumPp += sm.Pp[n];
-    if (!sm.has_child[n]) {
+    if (all_nodes || !sm.has_child[n]) {
       ++leaves;
       mx = fmax(mx, sm.Lc[n]);
       sumL += sm.Lc[n];
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_reward_kernel(RewardAr
   } else {
     double se = 0.0;
     for (int n = lane; n < g; n += 32)
-      if (!sm.has_child[n]) se += exp(eta * (sm.Lc[n] - mx));
+      if (all_nodes || !sm.has_child[n]) se += exp(eta * (sm.Lc[n] - mx));
     se = warp_sum_f64(se);
     reward = (eta * mx + log(se)) / eta;
   }

@@ -62,3 +62,22 @@ def test_invalid_arguments_are_refused_without_a_device(repo_root):
     with pytest.raises(gto.GtoError) as e:
         gto.gto_create(gto.make_config(8, 3, 12, 12, 8, 512, 512, "f32"), 0)   # k*k > 128
     assert e.value.code == 2
+
+
+def test_sample_groups_matches_the_oracle_on_the_host(repo_root):
+    """Host logic of SampleGroups (Algorithm 1, Eq. 6-7): the library against the oracle."""
+    import numpy as np
+    import pytest
+    from oracle import gto_oracle as orc
+    from paper_2509_22134_b200 import binding as gto
+    rng = np.random.default_rng(3)
+    for _ in range(300):
+        s, m = int(rng.integers(1, 400)), int(rng.integers(1, 33))
+        K = int(rng.integers(0, s // m + 1))
+        u = rng.random(K)
+        assert gto.gto_sample_groups(s, m, K, u) == orc.sample_groups(s, m, K, u)
+    assert gto.gto_sample_groups(2048, 8, 16, [0.999999] * 16) == [2048 - 128 + 1 + 8 * i for i in range(16)]
+    with pytest.raises(gto.GtoError):
+        gto.gto_sample_groups(10, 4, 3, [0.1, 0.2, 0.3])          # K*m > s
+    with pytest.raises(gto.GtoError):
+        gto.gto_sample_groups(10, 4, 1, [1.0])                    # not in [0, 1)

@@ -121,3 +121,38 @@ def test_ratio_is_one_when_old_equals_current_and_clip_edges():
     # not clipped in the pessimistic direction: A > 0 with s < 1-eps stays active
     sur = orc.clipped_surrogate(pl, old, [2, 1], [-1.0, 1.0], 2, eps=0.2)
     assert sur["active"].all()
+
+
+def test_sample_groups_respects_the_constraints_and_is_uniform_over_placements():
+    """Eq. 6-7: 1 <= t_k <= s - m + 1, t_{k+1} >= t_k + m.  Brute force on a tiny case: every
+    admissible placement is hit equally often when the uniforms sweep a fine grid."""
+    import itertools
+    s, m, K = 9, 2, 3
+    placements = [t for t in itertools.combinations(range(1, s - m + 2), K)
+                  if all(t[i + 1] >= t[i] + m for i in range(K - 1))]
+    counts = {t: 0 for t in placements}
+    n = s - K * m + 1
+    grid = [(i + 0.5) / n for i in range(n)]
+    for u in itertools.product(grid, repeat=K):
+        t = tuple(orc.sample_groups(s, m, K, u))
+        assert t in counts
+        counts[t] += 1
+    # sorted K-multisets of n gap values: each placement corresponds to one multiset; the
+    # number of orderings differs between multisets, so compare with the multinomial count
+    from math import factorial
+    from collections import Counter
+    for t, c in counts.items():
+        gaps = [t[i] - 1 - i * m for i in range(K)]
+        perms = factorial(K)
+        for rep in Counter(gaps).values():
+            perms //= factorial(rep)
+        assert c == perms
+    assert orc.sample_groups(16, 8, 2, [0.3, 0.9]) == [1, 9]       # no slack: the partition
+    assert orc.sample_groups(10, 4, 0, []) == []
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        s_, m_ = int(rng.integers(8, 300)), int(rng.integers(1, 9))
+        K_ = int(rng.integers(0, s_ // m_ + 1))
+        t = orc.sample_groups(s_, m_, K_, rng.random(K_))
+        assert all(1 <= x <= s_ - m_ + 1 for x in t)
+        assert all(t[i + 1] >= t[i] + m_ for i in range(len(t) - 1))

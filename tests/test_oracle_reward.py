@@ -194,3 +194,23 @@ def test_walk_stops_at_unexpanded_node_and_on_mismatch():
     target[0] = 0
     target[0, 2] = 9        # greedy token not among the root's children
     assert orc.longest_accepted(tree, target)["nodes"] == []
+
+
+def test_all_nodes_variant_sums_over_every_root_to_node_sequence():
+    """Independent restatement: walk every node's path with explicit products."""
+    draft, target, tree = tiny_case(11, V=6, D=4, k=3, g=12)
+    p, _ = orc.target_node_probs(tree, target)
+    Ls = []
+    for n in range(tree.g):
+        chain, x = [], n
+        while x >= 0:
+            chain.append(x)
+            x = int(tree.parent[x])
+        chain.reverse()
+        Ls.append(sum(np.prod([p[a] for a in chain[:j + 1]]) for j in range(len(chain))))
+    got = orc.tree_reward(tree, p, eta=1.3, all_nodes=True)
+    assert got["r"] == pytest.approx(logsumexp(1.3 * np.array(Ls)) / 1.3, rel=1e-12)
+    assert len(got["leaves"]) == tree.g
+    assert got["r"] >= orc.tree_reward(tree, p, eta=1.3)["r"]     # a superset of sequences
+    assert orc.tree_reward(tree, p, agg=orc.AGG_MAX, all_nodes=True)["r"] == \
+        orc.tree_reward(tree, p, agg=orc.AGG_MAX)["r"]            # the longest paths end in leaves

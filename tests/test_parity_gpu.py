@@ -67,6 +67,27 @@ def test_variants_max_mean_unbiased_nodebias(harness):
         harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(agg=oagg))
     p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_STD_UNBIASED | gto.GTO_FLAG_NO_DEBIAS)
     harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(unbiased=True, debias=False))
+    p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_SEQ_ALL_NODES)
+    rep = harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(all_nodes=True))
+    assert int(p.reward["n_leaves"].min()) == w.g
+
+
+@pytest.mark.parametrize("D,g", [(6, 50), (6, 70), (7, 50), (7, 70), (8, 50), (8, 60), (8, 70)])
+def test_tree_configuration_sweep(harness, D, g):
+    """Depth x node-budget grid of the tree-configuration ablation (App. E), top-k 10."""
+    w = synth.Workload("sweep", B=8, V_draft=8192, V_target=8192, D=D, k=10, g=g, seed=100 * D + g)
+    p, data = harness.run_pass(w, DEV)
+    harness.check_against_oracle(w, p, data, groups=[0])
+
+
+@pytest.mark.parametrize("m", [1, 4, 16, 32])
+def test_group_size_sweep(harness, m):
+    """Group sizes of the group-size ablation (Sec. 4.2); m = 1 gives zero advantages."""
+    w = synth.Workload("msweep", B=32, V_draft=2048, V_target=2048, D=4, k=4, g=20, m=m, seed=40 + m)
+    p, data = harness.run_pass(w, DEV)
+    harness.check_against_oracle(w, p, data, groups=list(range(w.B // m)))
+    if m == 1:
+        assert bool((p.stats["adv"] == 0).all()) and bool((p.grad == 0).all())
 
 
 def test_grad_live_rows_flag_leaves_the_other_rows_untouched(harness):
