@@ -46,13 +46,31 @@ struct TreeSmem {
 // Entries of a descending list that come before x; equal keys come before x iff `ties_first`.
 __device__ __forceinline__ int count_ahead(const uint64_t* list, int n, uint64_t x,
                                            bool ties_first) {
+  // x + 1 turns "y >= x" into "y > x": keys of finite scores never reach ~0
+  const uint64_t bound = ties_first ? x : x + 1;  // ahead iff y >= bound
   int lo = 0, hi = n;
   while (lo < hi) {
     const int mid = (lo + hi) >> 1;
-    const uint64_t y = list[mid];
-    if (y > x || (y == x && ties_first)) lo = mid + 1; else hi = mid;
+    if (list[mid] >= bound) lo = mid + 1; else hi = mid;
   }
   return lo;
+}
+
+// Same for a list of compile-time length N: a fixed number of branch-free steps (the answer
+// is built bit by bit from the top).
+template <int N>
+__device__ __forceinline__ int count_ahead_fixed(const uint64_t* list, uint64_t x,
+                                                 bool ties_first) {
+  const uint64_t bound = ties_first ? x : x + 1;
+  constexpr int kTopBit = N >= 16 ? 16 : N >= 8 ? 8 : N >= 4 ? 4 : N >= 2 ? 2 : 1;
+  static_assert(N < 32, "step table");
+  int pos = 0;  // entries [0, pos) are ahead
+#pragma unroll
+  for (int step = kTopBit; step > 0; step >>= 1) {
+    const int cand = pos + step;
+    if (cand <= N && list[cand - 1] >= bound) pos = cand;
+  }
+  return pos;
 }
 
 __device__ __forceinline__ int bits_below(const unsigned (&m)[kMaskWords], int q) {
@@ -65,12 +83,13 @@ __device__ __forceinline__ int bits_below(const unsigned (&m)[kMaskWords], int q
   return n;
 }
 
+template <int K>  // top-k known at compile time, or 0
 __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs a) {
   extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ TreeSmem sm;
   const int tid = threadIdx.x;
   const int tree = blockIdx.x;
-  const int D = a.D, k = a.k, g = a.g, R = a.R, kk = a.k * a.k;
+  const int D = a.D, k = K > 0 ? K : a.k, g = a.g, R = a.R, kk = k * k;
   const int P = k + (D - 1) * kk;
   uint64_t* skey = reinterpret_cast<uint64_t*>(dyn);       // [P] every layer, sorted
   uint8_t* sq = reinterpret_cast<uint8_t*>(skey + P);      // [P] candidate index at that rank
@@ -109,8 +128,14 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
     __syncthreads();
     if (tid < kk) {
       int rank = c;  // the children of one parent are in order already
-      for (int jp = 0; jp < k; ++jp)
-        if (jp != j) rank += count_ahead(&sm.ukey[jp * k], k, key, jp < j);
+      if constexpr (K > 0) {
+#pragma unroll
+        for (int jp = 0; jp < K; ++jp)
+          if (jp != j) rank += count_ahead_fixed<K>(&sm.ukey[jp * K], key, jp < j);
+      } else {
+        for (int jp = 0; jp < k; ++jp)
+          if (jp != j) rank += count_ahead(&sm.ukey[jp * k], k, key, jp < j);
+      }
       skey[base + rank] = key;
       sq[base + rank] = static_cast<uint8_t>(tid);
       if (d < D && rank < k) {
@@ -210,7 +235,10 @@ cudaError_t launch_tree_build(const TreeBuildArgs& a, cudaStream_t stream, int64
   if (a.n_trees <= 0) return cudaSuccess;
   const int P = a.k + (a.D - 1) * a.k * a.k;
   const size_t dyn = static_cast<size_t>(P) * (sizeof(uint64_t) + 1);
-  tree_build_kernel<<<a.n_trees, kTreeThreads, dyn, stream>>>(a);
+  if (a.k == 10)
+    tree_build_kernel<10><<<a.n_trees, kTreeThreads, dyn, stream>>>(a);  // the paper's top-k
+  else
+    tree_build_kernel<0><<<a.n_trees, kTreeThreads, dyn, stream>>>(a);
   ++*launches;
   return cudaGetLastError();
 }
