@@ -62,8 +62,9 @@ template <int N>
 __device__ __forceinline__ int count_ahead_fixed(const uint64_t* list, uint64_t x,
                                                  bool ties_first) {
   const uint64_t bound = ties_first ? x : x + 1;
-  constexpr int kTopBit = N >= 16 ? 16 : N >= 8 ? 8 : N >= 4 ? 4 : N >= 2 ? 2 : 1;
-  static_assert(N < 32, "step table");
+  constexpr int kTopBit = N >= 128 ? 128 : N >= 64 ? 64 : N >= 32 ? 32 : N >= 16 ? 16
+                          : N >= 8 ? 8 : N >= 4 ? 4 : N >= 2 ? 2 : 1;
+  static_assert(N < 256, "step table");
   int pos = 0;  // entries [0, pos) are ahead
 #pragma unroll
   for (int step = kTopBit; step > 0; step >>= 1) {
@@ -92,14 +93,22 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
   const int D = a.D, k = K > 0 ? K : a.k, g = a.g, R = a.R, kk = k * k;
   const int P = k + (D - 1) * kk;
   uint64_t* skey = reinterpret_cast<uint64_t*>(dyn);       // [P] every layer, sorted
-  uint8_t* sq = reinterpret_cast<uint8_t*>(skey + P);      // [P] candidate index at that rank
-  const double* lse = a.row_lse + static_cast<size_t>(tree) * R;
+  double* lse = reinterpret_cast<double*>(skey + P);        // [R] staged row log-sum-exps
+  float* top_z = reinterpret_cast<float*>(lse + R);        // [R*k] staged top-k logits
+  uint8_t* sq = reinterpret_cast<uint8_t*>(top_z + R * k); // [P] candidate index at that rank
   const int32_t* top_id = a.top_id + static_cast<size_t>(tree) * R * k;
-  const float* top_z = a.top_z + static_cast<size_t>(tree) * R * k;
+  {
+    // stage the tree's tables once: the layers then depend on shared memory only
+    const double* g_lse = a.row_lse + static_cast<size_t>(tree) * R;
+    const float* g_z = a.top_z + static_cast<size_t>(tree) * R * k;
+    for (int i = tid; i < R; i += kTreeThreads) lse[i] = g_lse[i];
+    for (int i = tid; i < R * k; i += kTreeThreads) top_z[i] = g_z[i];
+  }
   auto list_off = [&](int l) { return l == 0 ? 0 : k + (l - 1) * kk; };  // = pool index base
   auto list_len = [&](int l) { return l == 0 ? k : kk; };
 
   if (tid < D * kMaskWords) (&sm.selmask[0][0])[tid] = 0;
+  __syncthreads();
   // ---- depth 1: the root's k best tokens, already in rank order = pool order
   if (tid < k) {
     const double sc = static_cast<double>(top_z[tid]) - lse[0];
@@ -166,8 +175,14 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
     item(t, l, r);
     const uint64_t x = skey[list_off(l) + r];
     int rank = r;
-    for (int lp = 0; lp < D && rank < g; ++lp)
-      if (lp != l) rank += count_ahead(skey + list_off(lp), list_len(lp), x, lp < l);
+    if constexpr (K > 0) {
+      if (l != 0) rank += count_ahead_fixed<K>(skey, x, true);
+      for (int lp = 1; lp < D && rank < g; ++lp)
+        if (lp != l) rank += count_ahead_fixed<K * K>(skey + list_off(lp), x, lp < l);
+    } else {
+      for (int lp = 0; lp < D && rank < g; ++lp)
+        if (lp != l) rank += count_ahead(skey + list_off(lp), list_len(lp), x, lp < l);
+    }
     if (rank < g) {
       const int q = sq[list_off(l) + r];
       atomicOr(&sm.selmask[l][q >> 5], 1u << (q & 31));
@@ -234,7 +249,9 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
 cudaError_t launch_tree_build(const TreeBuildArgs& a, cudaStream_t stream, int64_t* launches) {
   if (a.n_trees <= 0) return cudaSuccess;
   const int P = a.k + (a.D - 1) * a.k * a.k;
-  const size_t dyn = static_cast<size_t>(P) * (sizeof(uint64_t) + 1);
+  const int R = 1 + (a.D - 1) * a.k;
+  const size_t dyn = static_cast<size_t>(P) * (sizeof(uint64_t) + 1) + R * sizeof(double) +
+                     static_cast<size_t>(R) * a.k * sizeof(float);
   if (a.k == 10)
     tree_build_kernel<10><<<a.n_trees, kTreeThreads, dyn, stream>>>(a);  // the paper's top-k
   else
