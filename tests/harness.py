@@ -36,6 +36,8 @@ def run_pass(w: synth.Workload, device="cuda:0", data=None, **kw):
     if data is None:
         data = synth.generate(w, device)
     p = GtoPass(w, device, **kw)
+    if kw.get("flags", 0) & 4:      # GTO_FLAG_GRAD_LIVE_ROWS: the other rows are the caller's
+        p.grad.zero_()
     p.build_tree(data["draft"])
     p.tree_reward(data["target"], data["d2t"])
     p.set_old_logp_from_path()
