@@ -31,6 +31,9 @@ def test_config0_all_positions(harness):
     (33000, 2, 10, 60, 8, "bf16"),
     (2048, 7, 11, 128, 8, "bf16"),    # compiled limits: k*k = 121, g = 128
     (512, 1, 8, 5, 8, "f32"),         # depth 1: the root row only
+    (256, 2, 3, 12, 8, "f32"),        # g = P: the whole candidate pool is kept
+    (1024, 16, 2, 62, 8, "bf16"),     # compiled depth limit, g = P = 62
+    (64, 3, 8, 40, 8, "bf16"),        # k = V / 8: one vector of the row per thread at most
 ])
 def test_small_shapes(harness, V, D, k, g, B, dtype):
     w = synth.Workload("t", B=B, V_draft=V, V_target=V, D=D, k=k, g=g, dtype=dtype, seed=V + D)
