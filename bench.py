@@ -354,10 +354,10 @@ def run_gpu(args, w, rank, world, local_rank):
 
 
 def run_e2e(args, w, dev, b0, world):
-    """The same pass through the same C-ABI calls with the logits in pinned HOST memory:
-    every step copies its positions' draft and target rows (and the old-policy
-    log-probabilities) to the device, runs the three calls and reads the losses, rewards,
-    advantages and accepted paths back.  The gradient stays on the device, where the
+    """The same pass through the C ABI with the logits in pinned HOST memory: every step
+    copies its positions' draft rows and the old-policy log-probabilities to the device,
+    builds the trees, copies the target rows the trees need (gto_tree_reward_host), and
+    reads the losses, rewards, advantages and accepted paths back.  The gradient stays on the device, where the
     draft model's backward pass consumes it."""
     from paper_2509_22134_b200 import synth
     from paper_2509_22134_b200.runner import GtoPass
@@ -375,14 +375,19 @@ def run_e2e(args, w, dev, b0, world):
             "reward": p.reward["reward"], "path_len": p.reward["path_len"],
             "path_row": p.reward["path_row"], "path_token": p.reward["path_token"]}
     back_host = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in back.items()}
-    h2d = sum(t.numel() * t.element_size() for t in host.values()) + old_host.numel() * 4
+    h2d_fixed = host["draft"].numel() * host["draft"].element_size() + old_host.numel() * 4
+    row_bytes = we.V_target * we.elem_bytes
     d2h = sum(t.numel() * t.element_size() for t in back.values())
+
+    rows = [0]
 
     def step():
         data["draft"].copy_(host["draft"], non_blocking=True)
-        data["target"].copy_(host["target"], non_blocking=True)
         p.old_logp.copy_(old_host, non_blocking=True)
-        p.step(data["draft"], data["target"], data["d2t"])
+        p.build_tree(data["draft"])
+        # only the target rows the trees need cross the bus (gto_tree_reward_host)
+        rows[0] = p.tree_reward_host(host["target"], data["target"], data["d2t"])
+        p.surrogate_grad(data["draft"])
         for k, v in back.items():
             back_host[k].copy_(v, non_blocking=True)
         torch.cuda.current_stream(dev).synchronize()       # the caller reads the results
@@ -403,6 +408,8 @@ def run_e2e(args, w, dev, b0, world):
     p.close()
     del data, host
     torch.cuda.empty_cache()
+    h2d = h2d_fixed + rows[0] * row_bytes   # + the row list read back (counted in d2h)
+    d2h += 4 * (we.G * we.B * we.R + 1)
     return {"ms": ms, "positions": we.B * steps, "h2d": h2d, "d2h": d2h,
             "positions_per_step": we.B, "steps": steps}
 

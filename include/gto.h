@@ -14,7 +14,8 @@
  * Logits are bf16 or fp32, row-major, contiguous; V_draft and V_target must make a row a
  * multiple of 16 bytes.  All pointers in the structs below are DEVICE pointers owned by
  * the caller, 16-byte aligned, dense row-major with the shapes given.  The library
- * allocates device memory only in gto_create (its workspace) and keeps no caller pointer
+ * allocates memory only in gto_create (its device workspace and a page-locked host copy of
+ * the row list for gto_tree_reward_host) and keeps no caller pointer
  * after a call returns.  Calls enqueue work on `stream` (a cudaStream_t passed as void*)
  * and return without synchronising; argument errors are returned at once and launch
  * nothing.  Data faults (a non-finite row sum, a bounded wait that ran out) are recorded
@@ -167,6 +168,19 @@ gto_status gto_build_tree_noalloc(const gto_config* cfg, int device, const void*
  * V_draft == V_target.  Writes every array of *out. */
 gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* target_logits,
                            const int32_t* d2t, const gto_reward* out, void* stream);
+
+/* gto_tree_reward for target logits that live in HOST memory (Eq. 3-5 and Sec. 3.2 as
+ * above).  Only the target rows that are the context of a selected node are needed
+ * (about a fifth of them at the paper's tree shape), so only those cross the bus: the call
+ * builds the row list on the device, reads it back (it SYNCHRONISES `stream` once), copies
+ * each run of adjacent needed rows from target_host to the same offset of target_dev, and
+ * then proceeds as gto_tree_reward on target_dev.  target_host: HOST [G,B,R,V_target],
+ * should be page-locked for the copies to be asynchronous; target_dev: DEVICE scratch of the
+ * same shape owned by the caller, rows that are not needed are left untouched.
+ * *rows_copied (optional, host) receives the number of rows copied. */
+gto_status gto_tree_reward_host(gto_ctx* ctx, const gto_tree* tree, const void* target_host,
+                                void* target_dev, const int32_t* d2t, const gto_reward* out,
+                                void* stream, int64_t* rows_copied);
 
 /* Eq. 9-12 and the derivative of the summed group losses with respect to the draft logits:
  * grad[b,j,:] = coeff_b * (onehot(path_token[b,j]) - softmax(draft row path_row[b,j] of

@@ -66,6 +66,9 @@ _lib.gto_build_tree_noalloc.argtypes = [ctypes.POINTER(gto_config), ctypes.c_int
                                         ctypes.POINTER(gto_tree), _vp]
 _lib.gto_build_tree_noalloc.restype = ctypes.c_int
 _lib.gto_tree_reward.argtypes = [_vp, ctypes.POINTER(gto_tree), _vp, _vp, ctypes.POINTER(gto_reward), _vp]
+_lib.gto_tree_reward_host.argtypes = [_vp, ctypes.POINTER(gto_tree), _vp, _vp, _vp,
+                                      ctypes.POINTER(gto_reward), _vp, ctypes.POINTER(ctypes.c_int64)]
+_lib.gto_tree_reward_host.restype = ctypes.c_int
 _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ctypes.POINTER(gto_reward),
                                           _vp, _vp, ctypes.POINTER(gto_grad_stats), _vp]
 _lib.gto_token_loss.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(gto_tree), ctypes.c_float, _vp,
@@ -185,6 +188,24 @@ def gto_tree_reward(ctx: int, tree: dict, target: torch.Tensor, d2t, reward: dic
                                 _stream_ptr(stream)), "gto_tree_reward")
 
 
+def gto_tree_reward_host(ctx: int, tree: dict, target_host: torch.Tensor, target_dev: torch.Tensor,
+                         d2t, reward: dict, stream=None) -> int:
+    """gto_tree_reward with the target logits in (pinned) host memory: copies only the
+    needed rows into target_dev.  Returns the number of rows copied."""
+    assert not target_host.is_cuda and target_host.is_contiguous()
+    assert target_dev.is_cuda and target_dev.is_contiguous()
+    assert target_host.shape == target_dev.shape and target_host.dtype == target_dev.dtype
+    if d2t is not None:
+        assert d2t.is_cuda and d2t.dtype == torch.int32 and d2t.is_contiguous()
+    t = _fill(gto_tree, _TREE_FIELDS, tree)
+    r = _fill(gto_reward, _REWARD_FIELDS, reward)
+    n = ctypes.c_int64(0)
+    _check(_lib.gto_tree_reward_host(ctx, ctypes.byref(t), target_host.data_ptr(), target_dev.data_ptr(),
+                                     None if d2t is None else d2t.data_ptr(), ctypes.byref(r),
+                                     _stream_ptr(stream), ctypes.byref(n)), "gto_tree_reward_host")
+    return int(n.value)
+
+
 def gto_group_surrogate_grad(ctx: int, draft: torch.Tensor, tree: dict, reward: dict,
                              old_logp: torch.Tensor, grad: torch.Tensor, stats: dict, stream=None):
     assert old_logp.is_cuda and old_logp.dtype == torch.float32 and old_logp.is_contiguous()
@@ -252,4 +273,4 @@ def gto_kernel_times(ctx: int, stream=None) -> dict:
 
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
            "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
-           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss", "gto_sample_groups"]
+           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss", "gto_sample_groups", "gto_tree_reward_host"]

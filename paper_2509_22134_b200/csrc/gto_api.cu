@@ -17,6 +17,8 @@ struct gto_ctx {
   int32_t* list;      // [G*B*R] needed target rows
   int32_t* list_count;
   int32_t* status;
+  int32_t* h_list;    // page-locked host copy of the work list: [0] = count, then the rows
+  int64_t last_host_rows;
   int64_t launches;
   bool timing;
   struct Span { cudaEvent_t t0, t1; int kernel; };
@@ -124,6 +126,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->R = R;
   ctx->P = static_cast<int>(P);
   ctx->launches = 0;
+  ctx->last_host_rows = 0;
   ctx->timing = false;
   ctx->spans_used = 0;
   size_t off = 0;
@@ -142,10 +145,12 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->list = reinterpret_cast<int32_t*>(ctx->ws + o_list);
   ctx->list_count = reinterpret_cast<int32_t*>(ctx->ws + o_cnt);
   ctx->status = reinterpret_cast<int32_t*>(ctx->ws + o_st);
-  if (cudaMemset(ctx->ws + o_cnt, 0, 512) != cudaSuccess) {
+  if (cudaMemset(ctx->ws + o_cnt, 0, 512) != cudaSuccess ||
+      cudaMallocHost(&ctx->h_list, (rows + 1) * sizeof(int32_t)) != cudaSuccess) {
+    cudaGetLastError();
     cudaFree(ctx->ws);
     delete ctx;
-    return GTO_ERR_CUDA;
+    return GTO_ERR_WORKSPACE;
   }
   *out = ctx;
   return GTO_OK;
@@ -158,6 +163,7 @@ gto_status gto_destroy(gto_ctx* ctx) {
     cudaEventDestroy(sp.t0);
     cudaEventDestroy(sp.t1);
   }
+  cudaFreeHost(ctx->h_list);
   cudaError_t e = cudaFree(ctx->ws);
   delete ctx;
   return e == cudaSuccess ? GTO_OK : GTO_ERR_CUDA;
@@ -202,8 +208,13 @@ gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, 
   return GTO_OK;
 }
 
-gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* target,
-                           const int32_t* d2t, const gto_reward* out, void* stream) {
+namespace {
+
+// Shared body of gto_tree_reward and gto_tree_reward_host.  With `target_host` the needed
+// rows are first copied from there into `target` (device) at their own offsets.
+gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* target,
+                            const void* target_host, const int32_t* d2t, const gto_reward* out,
+                            void* stream) {
   if (!ctx || !tree || !target || !out || !aligned16(target) || !all_set(tree) || !all_set(out))
     return GTO_ERR_INVALID_ARG;
   const gto_config& c = ctx->cfg;
@@ -224,6 +235,31 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   {
     LaunchSpan span(ctx, GTO_K_REWARD_PLAN, s);
     if (gto::launch_reward_plan(p, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  }
+  if (target_host != nullptr) {
+    // the host needs the list: one synchronisation, then one copy per run of adjacent rows
+    const size_t list_bytes = static_cast<size_t>(n_trees) * ctx->R * sizeof(int32_t);
+    if (cudaMemcpyAsync(ctx->h_list, ctx->list_count, sizeof(int32_t), cudaMemcpyDeviceToHost, s) !=
+            cudaSuccess ||
+        cudaMemcpyAsync(ctx->h_list + 1, ctx->list, list_bytes, cudaMemcpyDeviceToHost, s) !=
+            cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+      return GTO_ERR_CUDA;
+    const int count = ctx->h_list[0];
+    int32_t* rows = ctx->h_list + 1;
+    std::sort(rows, rows + count);
+    const size_t row_bytes = static_cast<size_t>(c.V_target) * (c.logit_dtype == GTO_BF16 ? 2 : 4);
+    for (int i = 0; i < count;) {
+      int j = i + 1;
+      while (j < count && rows[j] == rows[j - 1] + 1) ++j;
+      const size_t off = static_cast<size_t>(rows[i]) * row_bytes;
+      if (cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(target)) + off,
+                          static_cast<const char*>(target_host) + off, (j - i) * row_bytes,
+                          cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return GTO_ERR_CUDA;
+      i = j;
+    }
+    ctx->last_host_rows = count;
   }
   gto::RowReduceArgs r{};
   r.logits = target;
@@ -257,6 +293,22 @@ gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* targe
   LaunchSpan span(ctx, GTO_K_TREE_REWARD, s);
   if (gto::launch_tree_reward(w, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;
+}
+
+}  // namespace
+
+gto_status gto_tree_reward(gto_ctx* ctx, const gto_tree* tree, const void* target,
+                           const int32_t* d2t, const gto_reward* out, void* stream) {
+  return tree_reward_impl(ctx, tree, target, nullptr, d2t, out, stream);
+}
+
+gto_status gto_tree_reward_host(gto_ctx* ctx, const gto_tree* tree, const void* target_host,
+                                void* target_dev, const int32_t* d2t, const gto_reward* out,
+                                void* stream, int64_t* rows_copied) {
+  if (!target_host) return GTO_ERR_INVALID_ARG;
+  gto_status st = tree_reward_impl(ctx, tree, target_dev, target_host, d2t, out, stream);
+  if (st == GTO_OK && rows_copied) *rows_copied = ctx->last_host_rows;
+  return st;
 }
 
 gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_tree* tree,

@@ -44,6 +44,10 @@ class GtoPass:
     def tree_reward(self, target, d2t, stream=None):
         gto.gto_tree_reward(self.ctx, self.tree, target, d2t, self.reward, stream)
 
+    def tree_reward_host(self, target_host, target_dev, d2t, stream=None) -> int:
+        return gto.gto_tree_reward_host(self.ctx, self.tree, target_host, target_dev, d2t, self.reward,
+                                        stream)
+
     def surrogate_grad(self, draft, stream=None):
         gto.gto_group_surrogate_grad(self.ctx, draft, self.tree, self.reward, self.old_logp,
                                      self.grad, self.stats, stream)

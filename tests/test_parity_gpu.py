@@ -144,6 +144,26 @@ def test_token_loss_matches_the_oracle(harness, kw):
         assert np.all(err <= 2e-3 * weight + 2.0 ** -8 * np.abs(weight * g)), (b, err.max())
 
 
+def test_reward_from_host_rows_copies_only_the_needed_rows(harness):
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.WORKLOADS[1].with_B(16)
+    p_ref, data = harness.run_pass(w, DEV)
+    p = GtoPass(w, DEV)
+    p.build_tree(data["draft"])
+    host = torch.empty(data["target"].shape, dtype=data["target"].dtype, pin_memory=True).copy_(data["target"])
+    scratch = torch.full_like(data["target"], float("nan"))
+    n = p.tree_reward_host(host, scratch, data["d2t"])
+    torch.cuda.synchronize()
+    needed = ~torch.isnan(p_ref.reward["row_lse_t"])
+    assert n == int(needed.sum()) and 0 < n < needed.numel()
+    copied = ~torch.isnan(scratch[..., 0].float())
+    assert torch.equal(copied, needed)                      # exactly the needed rows crossed
+    assert torch.equal(scratch[needed], data["target"][needed])
+    for name in p.reward:
+        a, b = p.reward[name], p_ref.reward[name]
+        assert torch.equal(torch.nan_to_num(a.double(), nan=-7.0), torch.nan_to_num(b.double(), nan=-7.0)), name
+
+
 def test_deterministic_integer_outputs(harness):
     w = synth.WORKLOADS[1].with_B(32)
     p1, data = harness.run_pass(w, DEV)
