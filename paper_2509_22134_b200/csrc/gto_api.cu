@@ -11,6 +11,7 @@ struct gto_ctx {
   gto_config cfg;
   int device;
   int R, P;
+  int row_grid_cap;   // CTAs for the listed-row pass: a few waves of the device
   char* ws;           // one allocation
   int32_t* top_id;    // [G*B*R, k] draft row top-k ids
   float* top_z;       // [G*B*R, k] draft row top-k logits
@@ -25,6 +26,10 @@ struct gto_ctx {
   std::vector<Span> spans;   // event pairs, reused across reads
   size_t spans_used;
 };
+
+#ifndef GTO_ROW_GRID_WAVES
+#define GTO_ROW_GRID_WAVES 16  // resident-CTA waves launched for the listed-row pass (measured best of 1..24)
+#endif
 
 namespace {
 
@@ -126,6 +131,15 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->R = R;
   ctx->P = static_cast<int>(P);
   ctx->launches = 0;
+  {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+      cudaGetLastError();
+      delete ctx;
+      return GTO_ERR_CUDA;
+    }
+    ctx->row_grid_cap = sms * 12 * GTO_ROW_GRID_WAVES;
+  }
   ctx->last_host_rows = 0;
   ctx->timing = false;
   ctx->spans_used = 0;
@@ -269,6 +283,7 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
   r.pad = 0;
   r.list = ctx->list;
   r.list_count = ctx->list_count;
+  r.grid_cap = ctx->row_grid_cap;
   r.n_rows = n_trees * ctx->R;
   r.k = 1;
   r.out_lse = out->row_lse_t;

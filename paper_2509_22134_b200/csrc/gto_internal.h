@@ -28,6 +28,7 @@ struct RowReduceArgs {
   int32_t* out_id;           // [trees*R, k]
   float* out_z;              // [trees*R, k] or null
   int32_t* status;           // device status word
+  int grid_cap;              // with list: most CTAs to launch (0 = one per possible entry)
 };
 cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64_t* launches);
 

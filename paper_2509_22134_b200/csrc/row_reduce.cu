@@ -83,26 +83,14 @@ __device__ __forceinline__ void push_candidates(RowSmem& sm, const uint4& v, int
   }
 }
 
+// One row by the whole CTA: row r of tree `tree`, outputs at index gid.
 template <typename T>
-__global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduceArgs a) {
+__device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, int gid, int tree,
+                                           int r) {
   constexpr int E = T::kPerVec;
-  __shared__ RowSmem sm;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
-
-  // rows come either from the work list (1-D grid) or as (row in tree, tree) = (x, y)
-  int gid, tree, r;
-  if (a.list != nullptr) {
-    if (blockIdx.x >= *a.list_count) return;
-    gid = a.list[blockIdx.x];
-    tree = a.pad != 0 ? gid / a.R : 0;  // a tensor without padding rows needs no split
-    r = gid - tree * a.R;
-  } else {
-    r = blockIdx.x;
-    tree = blockIdx.y;
-    gid = tree * a.R + r;
-  }
   const char* row =
       static_cast<const char*>(a.logits) + tensor_row(tree, r, a.R, a.pad) * a.V * T::kBytes;
   const int nvec = a.V / E;
@@ -319,11 +307,32 @@ __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduc
   }
 }
 
+// Rows come either as (row in tree, tree) = (blockIdx.x, blockIdx.y), one per CTA, or from
+// the work list, which a bounded 1-D grid walks with a stride: the list's length is known
+// on the device only, and a CTA per possible entry would launch ~100 000 CTAs that exit at
+// once (measured: 0.54 ns each, 53 us per launch at the paper's shapes).
+template <typename T>
+__global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduceArgs a) {
+  __shared__ RowSmem sm;
+  if (a.list == nullptr) {
+    reduce_row<T>(a, sm, blockIdx.y * a.R + blockIdx.x, blockIdx.y, blockIdx.x);
+    return;
+  }
+  const int count = *a.list_count;
+  for (int li = blockIdx.x; li < count; li += gridDim.x) {
+    const int gid = a.list[li];
+    const int tree = a.pad != 0 ? gid / a.R : 0;  // a tensor without padding rows needs no split
+    reduce_row<T>(a, sm, gid, tree, gid - tree * a.R);
+    __syncthreads();  // the row's shared state is read to the end before the next row starts
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64_t* launches) {
   if (a.n_rows <= 0) return cudaSuccess;
   dim3 grid(a.n_rows), block(kThreads);
+  if (a.list != nullptr && a.grid_cap > 0 && a.n_rows > a.grid_cap) grid = dim3(a.grid_cap);
   if (a.list == nullptr) {
     if (a.n_rows % a.R != 0 || a.n_rows / a.R > 65535) return cudaErrorInvalidValue;
     grid = dim3(a.R, a.n_rows / a.R);
