@@ -164,6 +164,37 @@ def test_reward_from_host_rows_copies_only_the_needed_rows(harness):
         assert torch.equal(torch.nan_to_num(a.double(), nan=-7.0), torch.nan_to_num(b.double(), nan=-7.0)), name
 
 
+def test_the_three_calls_can_be_captured_in_a_cuda_graph_and_replayed(harness):
+    """The calls only enqueue work on the given stream (no allocation, no synchronisation),
+    so a small, launch-bound batch can be replayed as one graph launch."""
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.WORKLOADS[1].with_B(16)
+    p_ref, data = harness.run_pass(w, DEV)
+    p = GtoPass(w, DEV)
+    p.old_logp.copy_(p_ref.old_logp)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        p.step(data["draft"], data["target"], data["d2t"])       # warm-up outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    for t in list(p.tree.values()) + list(p.reward.values()) + list(p.stats.values()) + [p.grad]:
+        t.view(torch.uint8).zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        p.step(data["draft"], data["target"], data["d2t"])
+    for _ in range(2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert p.status() == 0
+    for name in p.tree:
+        assert torch.equal(p.tree[name], p_ref.tree[name]), name
+    for name in ("reward", "path_len", "path_node", "path_logp", "node_L"):
+        assert torch.equal(p.reward[name], p_ref.reward[name]), name
+    assert torch.equal(p.stats["adv"], p_ref.stats["adv"])
+    assert torch.equal(p.grad, p_ref.grad)
+
+
 def test_deterministic_integer_outputs(harness):
     w = synth.WORKLOADS[1].with_B(32)
     p1, data = harness.run_pass(w, DEV)
