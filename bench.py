@@ -40,11 +40,11 @@ E2E_POSITIONS = 64          # positions per end-to-end step (host buffers of ~2.
 # entry is used only while the kernel source it was taken from is unchanged.
 NCU_TRAFFIC = {
     # kernel: (source file, sha256 of that file at capture time, bytes per row, V of the capture)
-    # from profiles/row_reduce_workload2_b64.md
+    # from the ncu capture summarised under profiles/ (row pass, workload 2 shapes at B = 64)
     "draft_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                   "9af7c0ab7759533b118e6bd7a2687fca4b0bf05d5b6a792af05b570b44e830a1", (512533248 + 8308480) / 7808, 32000),
+                   "fabd0bd90e6442d5051974c8a5dc0790380d78840a67d425e1109255ba330860", (510941696 + 3525120) / 7808, 32000),
     "target_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                    "9af7c0ab7759533b118e6bd7a2687fca4b0bf05d5b6a792af05b570b44e830a1", (429916160 + 4603136) / 1673, 128256),
+                    "fabd0bd90e6442d5051974c8a5dc0790380d78840a67d425e1109255ba330860", (429940224 + 3521024) / 1673, 128256),
 }
 
 
