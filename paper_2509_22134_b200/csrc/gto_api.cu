@@ -52,20 +52,24 @@ struct DeviceGuard {
 struct LaunchSpan {
   gto_ctx* c;
   cudaStream_t s;
-  gto_ctx::Span* span = nullptr;
+  long index = -1;  // into c->spans (an index survives the vector growing)
   LaunchSpan(gto_ctx* ctx, int kernel, cudaStream_t stream) : c(ctx), s(stream) {
     if (!c->timing) return;
     if (c->spans_used == c->spans.size()) {
       gto_ctx::Span n{};
-      if (cudaEventCreate(&n.t0) != cudaSuccess || cudaEventCreate(&n.t1) != cudaSuccess) return;
+      if (cudaEventCreate(&n.t0) != cudaSuccess) return;
+      if (cudaEventCreate(&n.t1) != cudaSuccess) {
+        cudaEventDestroy(n.t0);
+        return;
+      }
       c->spans.push_back(n);
     }
-    span = &c->spans[c->spans_used++];
-    span->kernel = kernel;
-    cudaEventRecord(span->t0, s);
+    index = static_cast<long>(c->spans_used++);
+    c->spans[index].kernel = kernel;
+    cudaEventRecord(c->spans[index].t0, s);
   }
   ~LaunchSpan() {
-    if (span) cudaEventRecord(span->t1, s);
+    if (index >= 0) cudaEventRecord(c->spans[index].t1, s);
   }
 };
 
