@@ -196,3 +196,25 @@ def test_fig1_greedy_leaf_is_pruned_by_a_better_sibling_path():
     assert " ".join(greedy) == pruned[0]
     # and it would have scored the printed 0.36
     assert abs(edges[("It", "is")] * edges[("It is", "a")] - conf["It is a"]) < 1e-12
+
+
+def test_context_rows_follow_the_input_layout():
+    """Row 0 is the root context, row 1 + (d-1)k + j the context reached through frontier slot j
+    of depth d (the layout of the target tensor [R, V] with R = 1 + (D-1)k): written out for
+    D = 3, k = 2."""
+    assert [orc.context_row(0, 0, 2)] + [orc.context_row(d, j, 2) for d in (1, 2) for j in (0, 1)] == \
+        [0, 1, 2, 3, 4]
+    D, k, V = 3, 2, 4
+    draft = np.full((D, k, V), -20.0)
+    draft[0, 0, [2, 1]] = [3.0, 2.0]            # root: token 2 (slot 0), token 1 (slot 1)
+    draft[1, 0, [0, 3]] = [1.0, 0.5]            # under slot 0 of depth 1
+    draft[1, 1, [3, 0]] = [1.0, 0.9]            # under slot 1 of depth 1
+    draft[2, 0, [1, 2]] = [0.2, 0.1]            # contexts of depth 2, slots 0 and 1
+    draft[2, 1, [1, 2]] = [0.2, 0.1]
+    tree = orc.build_tree(draft, D, k, 10)      # g = P: every candidate
+    assert list(tree.depth) == [1, 1, 2, 2, 2, 2, 3, 3, 3, 3]
+    assert list(tree.ctx_row) == [0, 0, 1, 1, 2, 2, 3, 3, 4, 4]
+    assert list(tree.token[:6]) == [2, 1, 0, 3, 3, 0]
+    # depth-2 frontier: the two best of the four by cumulative score are both under token 2
+    assert list(tree.slot[:6]) == [0, 1, 0, 1, -1, -1]
+    assert list(tree.parent) == [-1, -1, 0, 0, 1, 1, 2, 2, 3, 3]
