@@ -55,7 +55,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         list(ex.map(compile_one, jobs))
     objs = [os.path.join(OBJ, s.replace(".cu", ".o")) for s in SOURCES]
     if force or jobs or _stale(LIB, objs):
-        r = subprocess.run([_nvcc(), "-shared", "-o", LIB, *objs, "-cudart", "static"],
+        r = subprocess.run([_nvcc(), "-shared", "-o", LIB, *objs, "-cudart", "static", "-ldl"],
                            capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"link failed:\n{r.stderr}")

@@ -4,6 +4,8 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
@@ -71,6 +73,12 @@ struct LaunchSpan {
   ~LaunchSpan() {
     if (index >= 0) cudaEventRecord(c->spans[index].t1, s);
   }
+};
+
+// NVTX range around one library call (a no-op unless a profiler is attached).
+struct CallRange {
+  explicit CallRange(const char* name) { nvtxRangePushA(name); }
+  ~CallRange() { nvtxRangePop(); }
 };
 
 template <typename S>
@@ -188,6 +196,7 @@ gto_status gto_destroy(gto_ctx* ctx) {
 }
 
 gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, void* stream) {
+  CallRange range("gto_build_tree");
   if (!ctx || !draft || !out || !aligned16(draft) || !all_set(out)) return GTO_ERR_INVALID_ARG;
   DeviceGuard guard(ctx->device);
   if (!guard.ok) return GTO_ERR_CUDA;
@@ -233,6 +242,7 @@ namespace {
 gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* target,
                             const void* target_host, const int32_t* d2t, const gto_reward* out,
                             void* stream) {
+  CallRange range(target_host ? "gto_tree_reward_host" : "gto_tree_reward");
   if (!ctx || !tree || !target || !out || !aligned16(target) || !all_set(tree) || !all_set(out))
     return GTO_ERR_INVALID_ARG;
   const gto_config& c = ctx->cfg;
@@ -333,6 +343,7 @@ gto_status gto_tree_reward_host(gto_ctx* ctx, const gto_tree* tree, const void* 
 gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_tree* tree,
                                     const gto_reward* reward, const float* old_logp, void* grad,
                                     const gto_grad_stats* out, void* stream) {
+  CallRange range("gto_group_surrogate_grad");
   if (!ctx || !draft || !tree || !reward || !old_logp || !grad || !out || !aligned16(draft) ||
       !aligned16(grad) || !aligned16(old_logp) || !all_set(tree) || !all_set(reward) ||
       !all_set(out))
@@ -366,6 +377,7 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
 gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, const int32_t* d2t,
                           const gto_tree* tree, float weight, void* grad_root,
                           const gto_token_stats* out, void* stream) {
+  CallRange range("gto_token_loss");
   if (!ctx || !draft || !target || !tree || !grad_root || !out || !aligned16(draft) ||
       !aligned16(target) || !aligned16(grad_root) || !all_set(tree) || !all_set(out))
     return GTO_ERR_INVALID_ARG;
