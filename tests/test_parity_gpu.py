@@ -240,6 +240,22 @@ def test_baseline_configs_sampled_groups(harness, cfg_id, groups):
     p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS if cfg_id == 2 else 0)
     rep = harness.check_against_oracle(w, p, data, groups=groups)
     print(cfg_id, rep)
+    # rows sampled over the whole batch, one by one against the oracle
+    from oracle import gto_oracle as orc
+    rng = np.random.default_rng(cfg_id)
+    dview = data["draft"].view(w.G, w.B, w.D * w.k, w.V_draft)
+    lse_t = p.reward["row_lse_t"]
+    needed = torch.nonzero(~torch.isnan(lse_t)).cpu().numpy()
+    for _ in range(48):
+        t, b, r = int(rng.integers(w.G)), int(rng.integers(w.B)), int(rng.integers(w.R))
+        z = dview[t, b, 0 if r == 0 else w.k + r - 1].float().cpu().numpy()
+        want, _, _ = orc.lse_and_topk(z, w.k)
+        assert abs(float(p.tree["row_lse"][t, b, r]) - want) <= 2e-6, (t, b, r)
+        t, b, r = (int(x) for x in needed[int(rng.integers(len(needed)))])
+        z = data["target"][t, b, r].float().cpu().numpy().astype(np.float64)
+        want = float(np.max(z) + np.log(np.sum(np.exp(z - np.max(z)))))
+        assert abs(float(lse_t[t, b, r]) - want) <= 2e-6, (t, b, r)
+        assert int(p.reward["row_argmax_t"][t, b, r]) == orc.argmax_low(z)
     # every tree obeys the structural invariants, at any size
     par = p.tree["node_parent"]
     n = torch.arange(w.g, device=par.device)
