@@ -11,7 +11,8 @@
  *   target [G, B, R, V_target]     R = 1 + (D-1)*k; row 0 = root context, row
  *                                  1 + (d-1)*k + j = frontier slot j of depth d.
  *
- * Logits are bf16 or fp32, row-major, contiguous; V_draft and V_target must make a row a
+ * Logits are bf16, fp16 (the paper trains under FP16 autocast, App. B) or fp32, row-major,
+ * contiguous; V_draft and V_target must make a row a
  * multiple of 16 bytes.  All pointers in the structs below are DEVICE pointers owned by
  * the caller, 16-byte aligned, dense row-major with the shapes given.  The library
  * allocates memory only in gto_create (its device workspace and a page-locked host copy of
@@ -44,7 +45,7 @@ typedef enum {
   GTO_ERR_TOO_LARGE = 7    /* gto_build_tree_noalloc: batch exceeds the fixed scratch    */
 } gto_status;
 
-typedef enum { GTO_F32 = 0, GTO_BF16 = 1 } gto_dtype;
+typedef enum { GTO_F32 = 0, GTO_BF16 = 1, GTO_F16 = 2 } gto_dtype;
 
 /* Reward aggregation over the tree's sequences: Eq. 5 (log-sum-exp smooth max, the
  * default) or the two alternatives of the aggregation ablation in Sec. 4.2. */

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgto.so")
 
 GTO_OK = 0
-GTO_F32, GTO_BF16 = 0, 1
+GTO_F32, GTO_BF16, GTO_F16 = 0, 1, 2
 GTO_AGG_LSE, GTO_AGG_MAX, GTO_AGG_MEAN = 0, 1, 2
 GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS, GTO_FLAG_GRAD_LIVE_ROWS, GTO_FLAG_SEQ_ALL_NODES = 1, 2, 4, 8
 
@@ -121,7 +121,8 @@ def _fill(struct_type, fields, bufs: dict):
 
 def make_config(B, D, k, g, m, V_draft, V_target, dtype, G=2, eta=1.0, clip_eps=0.2,
                 std_delta=1e-6, grad_scale=1.0, reward_agg=GTO_AGG_LSE, flags=0) -> gto_config:
-    code = {torch.bfloat16: GTO_BF16, torch.float32: GTO_F32, "bf16": GTO_BF16, "f32": GTO_F32}[dtype]
+    code = {torch.bfloat16: GTO_BF16, torch.float32: GTO_F32, torch.float16: GTO_F16,
+            "bf16": GTO_BF16, "f32": GTO_F32, "f16": GTO_F16}[dtype]
     return gto_config(B, G, D, k, g, m, V_draft, V_target, code, reward_agg,
                       eta, clip_eps, std_delta, grad_scale, flags)
 

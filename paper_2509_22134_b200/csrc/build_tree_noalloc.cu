@@ -54,7 +54,7 @@ extern "C" gto_status gto_build_tree_noalloc(const gto_config* c, int device, co
   if (device < 0 || device >= kMaxDevices) return GTO_ERR_INVALID_ARG;
   if (c->B <= 0 || c->D <= 0 || c->k <= 0 || c->g <= 0 || c->V_draft <= 0)
     return GTO_ERR_INVALID_ARG;
-  if (c->logit_dtype != GTO_F32 && c->logit_dtype != GTO_BF16) return GTO_ERR_INVALID_ARG;
+  if (!gto::valid_dtype(c->logit_dtype)) return GTO_ERR_INVALID_ARG;
   if (c->k > c->V_draft) return GTO_ERR_INVALID_ARG;
   const int64_t P = c->k + static_cast<int64_t>(c->D - 1) * c->k * c->k;
   if (c->g > P) return GTO_ERR_INVALID_ARG;
@@ -62,7 +62,7 @@ extern "C" gto_status gto_build_tree_noalloc(const gto_config* c, int device, co
   if (c->k > gto::kMaxTopK || c->k * c->k > gto::kMaxLayer || c->g > gto::kMaxNodes ||
       c->D > gto::kMaxDepth)
     return GTO_ERR_UNSUPPORTED;
-  if ((static_cast<int64_t>(c->V_draft) * (c->logit_dtype == GTO_BF16 ? 2 : 4)) % 16)
+  if ((static_cast<int64_t>(c->V_draft) * gto::elem_bytes(c->logit_dtype)) % 16)
     return GTO_ERR_UNSUPPORTED;
   if (static_cast<int64_t>(c->G) * c->B > 65535) return GTO_ERR_UNSUPPORTED;
   const int R = 1 + (c->D - 1) * c->k;

@@ -114,7 +114,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   if (c->B <= 0 || c->D <= 0 || c->k <= 0 || c->g <= 0 || c->m <= 0 || c->V_draft <= 0 ||
       c->V_target <= 0)
     return GTO_ERR_INVALID_ARG;
-  if (c->logit_dtype != GTO_F32 && c->logit_dtype != GTO_BF16) return GTO_ERR_INVALID_ARG;
+  if (!gto::valid_dtype(c->logit_dtype)) return GTO_ERR_INVALID_ARG;
   if (c->reward_agg < GTO_AGG_LSE || c->reward_agg > GTO_AGG_MEAN) return GTO_ERR_INVALID_ARG;
   if (!(c->eta > 0.f) || !(c->clip_eps >= 0.f) || !(c->std_delta >= 0.f))
     return GTO_ERR_INVALID_ARG;
@@ -126,7 +126,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   if (c->k > gto::kMaxTopK || c->k * c->k > gto::kMaxLayer || c->g > gto::kMaxNodes ||
       c->D > gto::kMaxDepth)
     return GTO_ERR_UNSUPPORTED;
-  const int eb = c->logit_dtype == GTO_BF16 ? 2 : 4;
+  const int eb = gto::elem_bytes(c->logit_dtype);
   if ((static_cast<int64_t>(c->V_draft) * eb) % 16 || (static_cast<int64_t>(c->V_target) * eb) % 16)
     return GTO_ERR_UNSUPPORTED;
   const int R = 1 + (c->D - 1) * c->k;
@@ -276,7 +276,7 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
     const int count = ctx->h_list[0];
     int32_t* rows = ctx->h_list + 1;
     std::sort(rows, rows + count);
-    const size_t row_bytes = static_cast<size_t>(c.V_target) * (c.logit_dtype == GTO_BF16 ? 2 : 4);
+    const size_t row_bytes = static_cast<size_t>(c.V_target) * gto::elem_bytes(c.logit_dtype);
     for (int i = 0; i < count;) {
       int j = i + 1;
       while (j < count && rows[j] == rows[j - 1] + 1) ++j;

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -81,6 +82,48 @@ struct Bf16 {
   }
   __device__ static __forceinline__ float max_value(MaxAcc acc) {
     return fmaxf(__uint_as_float(acc << 16), __uint_as_float(acc & 0xffff0000u));
+  }
+};
+
+struct F16 {
+  static constexpr int kPerVec = 8;
+  static constexpr int kBytes = 2;
+  static constexpr uint32_t kNegInfWord = 0xfc00fc00u;
+  __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&w[q]));
+      f[2 * q] = p.x;
+      f[2 * q + 1] = p.y;
+    }
+  }
+  __device__ static __forceinline__ uint4 pack(const float (&f)[8]) {
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const __half2 h = __floats2half2_rn(f[2 * q], f[2 * q + 1]);
+      w[q] = *reinterpret_cast<const uint32_t*>(&h);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+  __device__ static __forceinline__ float load1(const void* base, size_t idx) {
+    return __half2float(reinterpret_cast<const __half*>(base)[idx]);
+  }
+  // Running maximum kept as two packed fp16 lanes.
+  using MaxAcc = uint32_t;
+  __device__ static __forceinline__ MaxAcc max_init() { return kNegInfWord; }
+  __device__ static __forceinline__ uint32_t max2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+  }
+  __device__ static __forceinline__ void max_update(MaxAcc& acc, const uint4& v) {
+    acc = max2(acc, max2(max2(v.x, v.y), max2(v.z, v.w)));
+  }
+  __device__ static __forceinline__ float max_value(MaxAcc acc) {
+    const float2 p = __half22float2(*reinterpret_cast<const __half2*>(&acc));
+    return fmaxf(p.x, p.y);
   }
 };
 

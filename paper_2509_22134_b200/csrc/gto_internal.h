@@ -8,6 +8,9 @@
 
 namespace gto {
 
+inline int elem_bytes(int dtype) { return dtype == GTO_F32 ? 4 : 2; }
+inline bool valid_dtype(int dtype) { return dtype == GTO_F32 || dtype == GTO_BF16 || dtype == GTO_F16; }
+
 constexpr int kMaxTopK = 16;       // per-row top-k the row kernel can hold
 constexpr int kMaxLayer = 128;     // k*k candidates per layer
 constexpr int kMaxNodes = 128;     // g

@@ -339,6 +339,8 @@ cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64
   }
   if (a.dtype == GTO_BF16)
     row_reduce_kernel<Bf16><<<grid, block, 0, stream>>>(a);
+  else if (a.dtype == GTO_F16)
+    row_reduce_kernel<F16><<<grid, block, 0, stream>>>(a);
   else
     row_reduce_kernel<F32><<<grid, block, 0, stream>>>(a);
   ++*launches;

@@ -125,13 +125,15 @@ cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* 
 }
 
 cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
-  int vec_per_row = a.V / (a.dtype == GTO_BF16 ? 8 : 4);
+  int vec_per_row = a.V / (16 / elem_bytes(a.dtype));
   int split = (vec_per_row + kGradThreads * 8 - 1) / (kGradThreads * 8);  // ~8 vectors/thread
   if (split < 1) split = 1;
   if (split > 64) split = 64;
   dim3 grid(a.B * a.D, split), block(kGradThreads);
   if (a.dtype == GTO_BF16)
     grad_rows_kernel<Bf16><<<grid, block, 0, stream>>>(a);
+  else if (a.dtype == GTO_F16)
+    grad_rows_kernel<F16><<<grid, block, 0, stream>>>(a);
   else
     grad_rows_kernel<F32><<<grid, block, 0, stream>>>(a);
   ++*launches;

@@ -150,6 +150,8 @@ cudaError_t launch_token_loss(const TokenLossArgs& a, cudaStream_t stream, int64
   if (a.B <= 0) return cudaSuccess;
   if (a.dtype == GTO_BF16)
     token_loss_kernel<Bf16><<<a.B, kTokThreads, 0, stream>>>(a);
+  else if (a.dtype == GTO_F16)
+    token_loss_kernel<F16><<<a.B, kTokThreads, 0, stream>>>(a);
   else
     token_loss_kernel<F32><<<a.B, kTokThreads, 0, stream>>>(a);
   ++*launches;

@@ -204,6 +204,8 @@ cudaError_t launch_tree_reward(const RewardArgs& a, cudaStream_t stream, int64_t
   dim3 grid((n_trees + kWarpsPerCta - 1) / kWarpsPerCta), block(kWarpsPerCta * 32);
   if (a.dtype == GTO_BF16)
     tree_reward_kernel<Bf16><<<grid, block, 0, stream>>>(a);
+  else if (a.dtype == GTO_F16)
+    tree_reward_kernel<F16><<<grid, block, 0, stream>>>(a);
   else
     tree_reward_kernel<F32><<<grid, block, 0, stream>>>(a);
   ++*launches;

@@ -110,7 +110,7 @@ class Workload:
     g: int
     G: int = 2
     m: int = 8
-    dtype: str = "bf16"          # "bf16" or "f32"
+    dtype: str = "bf16"          # "bf16", "f16" or "f32"
     sigma_t: float = 2.5         # scale of the target base distribution
     boost: float = 8.0           # added to the seeded true token of every target row
     sigma_d: float = 0.7         # draft = target + N(0, sigma_d^2)
@@ -132,11 +132,11 @@ class Workload:
 
     @property
     def torch_dtype(self):
-        return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+        return {"bf16": torch.bfloat16, "f16": torch.float16, "f32": torch.float32}[self.dtype]
 
     @property
     def elem_bytes(self) -> int:
-        return 2 if self.dtype == "bf16" else 4
+        return 4 if self.dtype == "f32" else 2
 
     def with_B(self, B: int) -> "Workload":
         return replace(self, B=B)

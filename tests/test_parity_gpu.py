@@ -34,6 +34,8 @@ def test_config0_all_positions(harness):
     (256, 2, 3, 12, 8, "f32"),        # g = P: the whole candidate pool is kept
     (1024, 16, 2, 62, 8, "bf16"),     # compiled depth limit, g = P = 62
     (64, 3, 8, 40, 8, "bf16"),        # k = V / 8: one vector of the row per thread at most
+    (4104, 4, 3, 17, 16, "f16"),      # fp16 logits (the paper's autocast precision), ragged tail
+    (32000, 3, 10, 30, 8, "f16"),
 ])
 def test_small_shapes(harness, V, D, k, g, B, dtype):
     w = synth.Workload("t", B=B, V_draft=V, V_target=V, D=D, k=k, g=g, dtype=dtype, seed=V + D)
@@ -117,6 +119,7 @@ def test_grad_live_rows_flag_leaves_the_other_rows_untouched(harness):
     dict(B=16, V_draft=4104, V_target=4104, D=3, k=4, g=12, dtype="bf16", seed=21),
     dict(B=16, V_draft=2048, V_target=8200, D=3, k=4, g=12, dtype="bf16", seed=22),   # id map
     dict(B=8, V_draft=1000, V_target=1000, D=2, k=4, g=8, dtype="f32", seed=23),
+    dict(B=8, V_draft=2048, V_target=8200, D=2, k=4, g=8, dtype="f16", seed=25),
     dict(B=8, V_draft=32000, V_target=128256, D=2, k=10, g=20, dtype="bf16", seed=24),
 ])
 def test_token_loss_matches_the_oracle(harness, kw):
