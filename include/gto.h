@@ -54,6 +54,9 @@ typedef enum { GTO_AGG_LSE = 0, GTO_AGG_MAX = 1, GTO_AGG_MEAN = 2 } gto_agg;
 enum {
   GTO_FLAG_STD_UNBIASED = 1u, /* Eq. 10 with the sample std (divide by m-1)             */
   GTO_FLAG_NO_DEBIAS = 2u,    /* Eq. 9 switched off: R_i = r(T_i) (debiasing ablation)  */
+  GTO_FLAG_FORCE_ROW_SPLIT = 16u, /* always split a logit row over a thread-block cluster (the
+                                  library does so by itself where it pays: few, long rows);
+                                  for tests and tuning                                      */
   GTO_FLAG_SEQ_ALL_NODES = 8u, /* Eq. 5 over the root-to-node sequence of every selected node
                                   instead of the root-to-leaf sequences only                 */
   GTO_FLAG_GRAD_LIVE_ROWS = 4u /* gto_group_surrogate_grad writes only the rows that carry a

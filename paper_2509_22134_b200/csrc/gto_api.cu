@@ -14,6 +14,7 @@ struct gto_ctx {
   int device;
   int R, P;
   int row_grid_cap;   // CTAs for the listed-row pass: a few waves of the device
+  int row_split_rows;   // batches with at most this many rows may split every row over a cluster
   char* ws;           // one allocation
   int32_t* top_id;    // [G*B*R, k] draft row top-k ids
   float* top_z;       // [G*B*R, k] draft row top-k logits
@@ -29,6 +30,9 @@ struct gto_ctx {
   size_t spans_used;
 };
 
+#ifndef GTO_ROW_SPLIT_ROWS_PER_SM
+#define GTO_ROW_SPLIT_ROWS_PER_SM 6  // up to this many rows per SM, a row is split over a cluster
+#endif
 #ifndef GTO_ROW_GRID_WAVES
 #define GTO_ROW_GRID_WAVES 16  // resident-CTA waves launched for the listed-row pass (measured best of 1..24)
 #endif
@@ -80,6 +84,16 @@ struct CallRange {
   explicit CallRange(const char* name) { nvtxRangePushA(name); }
   ~CallRange() { nvtxRangePop(); }
 };
+
+// Rows are split over a cluster only where that was measured to pay: few rows (at most
+// GTO_ROW_SPLIT_ROWS_PER_SM per SM) that are long (slices of at least 32 KB).  At the paper's
+// shapes that is the target pass below 8 positions and 300 KB draft rows of small batches; 64 KB
+// draft rows are faster unsplit at any batch size (22 vs 46 us at 976 rows).
+int split_below(const gto_ctx* ctx, int n_rows, int V) {
+  const size_t row_bytes = static_cast<size_t>(V) * gto::elem_bytes(ctx->cfg.logit_dtype);
+  const bool pays = n_rows <= ctx->row_split_rows && row_bytes >= 4 * 32768;
+  return (pays || (ctx->cfg.flags & GTO_FLAG_FORCE_ROW_SPLIT)) ? n_rows : 0;
+}
 
 template <typename S>
 bool all_set(const S* s) {
@@ -151,6 +165,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
       return GTO_ERR_CUDA;
     }
     ctx->row_grid_cap = sms * 12 * GTO_ROW_GRID_WAVES;
+    ctx->row_split_rows = sms * GTO_ROW_SPLIT_ROWS_PER_SM;
   }
   ctx->last_host_rows = 0;
   ctx->timing = false;
@@ -216,6 +231,7 @@ gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, 
   r.out_id = ctx->top_id;
   r.out_z = ctx->top_z;
   r.status = ctx->status;
+  r.split_below = split_below(ctx, r.n_rows, r.V);
   {
     LaunchSpan span(ctx, GTO_K_DRAFT_ROWS, s);
     if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
@@ -304,6 +320,7 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
   r.out_id = out->row_argmax_t;
   r.out_z = nullptr;
   r.status = ctx->status;
+  r.split_below = split_below(ctx, r.n_rows, r.V);
   {
     LaunchSpan span(ctx, GTO_K_TARGET_ROWS, s);
     if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;

@@ -24,14 +24,23 @@
 // rank among the candidates is then counted directly.  A row with more candidates than the
 // buffer holds (massive ties) takes k exact arg-max rounds.
 //
+// Few rows (a small batch): one CTA per row leaves most SMs idle and a CTA alone is bound
+// by its own load latency, so the row is split over a thread-block cluster of kSplit CTAs,
+// each running the same procedure on a slice of the vocabulary; the cluster's first CTA then
+// reads the slices' partial sums and best keys through distributed shared memory and merges.
+//
 // The pass is bound by instruction issue as much as by HBM (one exponential per logit), so
 // the streaming loop keeps the running maximum packed (two bf16 lanes per instruction) and
 // warp maxima use the integer redux instruction on order-preserving keys.
+#include <cooperative_groups.h>
+
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
 namespace gto {
 namespace {
+
+namespace cg = cooperative_groups;
 
 #ifndef GTO_ROW_THREADS
 #define GTO_ROW_THREADS 128
@@ -52,6 +61,16 @@ constexpr float kRebase = 8.f;  // largest exponent argument before a thread mov
 
 static_assert(kMaxPer * kWarps <= 32, "one lane per kept maximum");
 constexpr uint32_t kKeyNegInf = 0x007fffffu;  // orderable(-inf): stands for "no element"
+
+constexpr int kSplit = 4;  // CTAs (one cluster) per row in the split variant
+
+// What one CTA of a split row hands to the cluster's first CTA.
+struct RowPartial {
+  double sum;                           // sum of 2^(z*log2e - ref) over the slice
+  float ref;
+  int n;                                // valid keys
+  unsigned long long key[kMaxTopK];     // the slice's best (value, id) keys, descending
+};
 
 struct RowSmem {
   uint32_t warp_top[kMaxPer * kWarps];  // each warp's largest thread maxima, as orderable keys
@@ -83,17 +102,34 @@ __device__ __forceinline__ void push_candidates(RowSmem& sm, const uint4& v, int
   }
 }
 
-// One row by the whole CTA: row r of tree `tree`, outputs at index gid.
-template <typename T>
+// lse = ref / log2e + ln2 * log2(sum): log2 of the fp64 total as exponent + log2f(mantissa in
+// [1,2)), so the fp32 logarithm's error stays below 1e-7.  A sum that is 0 (no terms), inf or
+// NaN gives a non-finite result, which the caller reports.
+__device__ __forceinline__ double lse_from_sum(float ref, double S) {
+  if (S > 0.0 && S < 1e300) {
+    int ex;
+    const double mant = frexp(S, &ex);  // S = mant * 2^ex, mant in [0.5, 1)
+    const double lg = static_cast<double>(ex - 1) +
+                      static_cast<double>(log2f(static_cast<float>(mant * 2.0)));
+    return static_cast<double>(ref) / static_cast<double>(kLog2e) + kLn2 * lg;
+  }
+  return (S == 0.0) ? -INFINITY : S;
+}
+
+// One row, or with SPLIT the slice [v_begin, v_begin + v_count) of its 16-byte vectors, by the
+// whole CTA: row r of tree `tree`.  Results go to the outputs at index gid, with SPLIT to *part.
+template <typename T, bool SPLIT>
 __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, int gid, int tree,
-                                           int r) {
+                                           int r, int v_begin, int v_count, RowPartial* part) {
   constexpr int E = T::kPerVec;
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
-  const char* row =
-      static_cast<const char*>(a.logits) + tensor_row(tree, r, a.R, a.pad) * a.V * T::kBytes;
-  const int nvec = a.V / E;
+  const char* row = static_cast<const char*>(a.logits) +
+                    tensor_row(tree, r, a.R, a.pad) * a.V * T::kBytes +
+                    (SPLIT ? static_cast<size_t>(v_begin) * 16 : 0);
+  const int nvec = SPLIT ? v_count : a.V / E;
+  const int vec0 = SPLIT ? v_begin : 0;  // vector index of the slice's first vector in the row
   const int k = a.k;
 
   // ---- pass 1: per-thread exponential sum; largest and second-largest batch maximum.
@@ -221,15 +257,17 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
       uint4 v[kUnroll];
       load_checked(v, i1);
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u)
-        push_candidates<T>(sm, v[u], tid + i1 * kBatchVecs + u * kThreads, tau);
+      for (int u = 0; u < kUnroll; ++u) {
+        const int i = tid + i1 * kBatchVecs + u * kThreads;
+        if (i < nvec) push_candidates<T>(sm, v[u], vec0 + i, tau);
+      }
     }
     unsigned todo = __ballot_sync(kFull, b2 >= tau);  // several batches: rescan the thread
     while (todo) {
       const int src = __ffs(todo) - 1;
       todo &= todo - 1;
       for (int i = warp * 32 + src + lane * kThreads; i < nvec; i += 32 * kThreads)
-        push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(i) * 16), i, tau);
+        push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(i) * 16), vec0 + i, tau);
     }
   }
   __syncthreads();
@@ -245,10 +283,15 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
       int rank = 0;
       for (int j = 0; j < n_cand; ++j) rank += sm.cand[j] > key ? 1 : 0;
       if (rank < k) {
-        out_id[rank] = key_id(key);
-        if (out_z) out_z[rank] = key_value(key);
+        if constexpr (SPLIT) {
+          part->key[rank] = key;
+        } else {
+          out_id[rank] = key_id(key);
+          if (out_z) out_z[rank] = key_value(key);
+        }
       }
     }
+    if (SPLIT && tid == 0) part->n = n_cand < k ? n_cand : k;
   } else {
     // ---- too many ties at tau: k exact arg-max rounds over the whole row
     if (tid == 0) sm.prev_key = ~0ull;
@@ -262,7 +305,7 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
         T::unpack(v, f);
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-          uint64_t key = make_key(f[e], i * E + e);
+          uint64_t key = make_key(f[e], (vec0 + i) * E + e);
           if (key < prev && key > best) best = key;
         }
       }
@@ -273,16 +316,20 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
         uint64_t b = 0;
         for (int w = 0; w < kWarps; ++w) b = sm.round_best[w] > b ? sm.round_best[w] : b;
         sm.prev_key = b;
-        out_id[round] = key_id(b);
-        if (out_z) out_z[round] = key_value(b);
+        if constexpr (SPLIT) {
+          part->key[round] = b;
+          part->n = k;
+        } else {
+          out_id[round] = key_id(b);
+          if (out_z) out_z[round] = key_value(b);
+        }
       }
       __syncthreads();
     }
   }
 
   // ---- row log-sum-exp: shift the warps' sums to a common reference (exact powers of two
-  //      times sums that carry 2^-22 already), then log2 of the fp64 total as exponent +
-  //      log2f(mantissa in [1,2)), so the fp32 logarithm's error stays below 1e-7
+  //      times sums that carry 2^-22 already) and add them in fp64
   if (tid == 0) {
     float Ref = -INFINITY;
     for (int w = 0; w < kWarps; ++w)
@@ -292,16 +339,53 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
       if (sm.warp_sum[w] != 0.f)
         S += static_cast<double>(sm.warp_sum[w]) *
              static_cast<double>(exp2f(sm.warp_ref[w] - Ref));
-    double lse;
-    if (S > 0.0 && S < 1e300) {
-      int ex;
-      const double mant = frexp(S, &ex);  // S = mant * 2^ex, mant in [0.5, 1)
-      const double lg = static_cast<double>(ex - 1) +
-                        static_cast<double>(log2f(static_cast<float>(mant * 2.0)));
-      lse = static_cast<double>(Ref) / static_cast<double>(kLog2e) + kLn2 * lg;
+    if constexpr (SPLIT) {
+      part->ref = Ref;
+      part->sum = S;
     } else {
-      lse = (S == 0.0) ? -INFINITY : S;  // no terms, inf or NaN: reported below
+      const double lse = lse_from_sum(Ref, S);
+      if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
+      a.out_lse[gid] = lse;
     }
+  }
+}
+
+// The first CTA of a cluster merges the slices of a split row: partial sums are shifted to
+// the largest reference; the row's top-k are the best k of the slices' best keys.
+template <typename T>
+__device__ __forceinline__ void merge_row(const RowReduceArgs& a, cg::cluster_group& cluster,
+                                          RowPartial* mine, int gid) {
+  const int tid = threadIdx.x;
+  const int k = a.k;
+  if (tid < kSplit * kMaxTopK) {
+    const RowPartial* own = cluster.map_shared_rank(mine, tid / kMaxTopK);
+    const int j = tid % kMaxTopK;
+    if (j < own->n) {
+      const uint64_t key = own->key[j];
+      int rank = 0;
+      for (int c = 0; c < kSplit; ++c) {
+        const RowPartial* pc = cluster.map_shared_rank(mine, c);
+        const int n = pc->n;
+        for (int q = 0; q < n; ++q) rank += pc->key[q] > key ? 1 : 0;
+      }
+      if (rank < k) {
+        a.out_id[static_cast<size_t>(gid) * k + rank] = key_id(key);
+        if (a.out_z) a.out_z[static_cast<size_t>(gid) * k + rank] = key_value(key);
+      }
+    }
+  }
+  if (tid == 0) {
+    float Ref = -INFINITY;
+    for (int c = 0; c < kSplit; ++c) {
+      const RowPartial* pc = cluster.map_shared_rank(mine, c);
+      if (pc->sum != 0.0) Ref = fmaxf(Ref, pc->ref);
+    }
+    double S = 0.0;
+    for (int c = 0; c < kSplit; ++c) {
+      const RowPartial* pc = cluster.map_shared_rank(mine, c);
+      if (pc->sum != 0.0) S += pc->sum * static_cast<double>(exp2f(pc->ref - Ref));
+    }
+    const double lse = lse_from_sum(Ref, S);
     if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
     a.out_lse[gid] = lse;
   }
@@ -315,15 +399,48 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduceArgs a) {
   __shared__ RowSmem sm;
   if (a.list == nullptr) {
-    reduce_row<T>(a, sm, blockIdx.y * a.R + blockIdx.x, blockIdx.y, blockIdx.x);
+    reduce_row<T, false>(a, sm, blockIdx.y * a.R + blockIdx.x, blockIdx.y, blockIdx.x, 0, 0, nullptr);
     return;
   }
   const int count = *a.list_count;
   for (int li = blockIdx.x; li < count; li += gridDim.x) {
     const int gid = a.list[li];
     const int tree = a.pad != 0 ? gid / a.R : 0;  // a tensor without padding rows needs no split
-    reduce_row<T>(a, sm, gid, tree, gid - tree * a.R);
+    reduce_row<T, false>(a, sm, gid, tree, gid - tree * a.R, 0, 0, nullptr);
     __syncthreads();  // the row's shared state is read to the end before the next row starts
+  }
+}
+
+// The same with every row split over a cluster of kSplit CTAs (grid.x counts CTAs: kSplit per
+// row or per list walker).
+template <typename T>
+__global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, kMinCtas)
+    row_reduce_split_kernel(RowReduceArgs a) {
+  __shared__ RowSmem sm;
+  __shared__ RowPartial part;
+  cg::cluster_group cluster = cg::this_cluster();
+  const int slice = static_cast<int>(cluster.block_rank());
+  const int nvec = a.V / T::kPerVec;
+  const int per_slice = (nvec + kSplit - 1) / kSplit;
+  const int v_begin = min(slice * per_slice, nvec);
+  const int v_count = min(per_slice, nvec - v_begin);
+  const int walker = blockIdx.x / kSplit, walkers = gridDim.x / kSplit;
+  const int count = a.list != nullptr ? *a.list_count : 1;
+  for (int li = a.list != nullptr ? walker : 0; li < count; li += walkers) {
+    int gid, tree, r;
+    if (a.list != nullptr) {
+      gid = a.list[li];
+      tree = a.pad != 0 ? gid / a.R : 0;
+      r = gid - tree * a.R;
+    } else {
+      r = walker;
+      tree = blockIdx.y;
+      gid = tree * a.R + r;
+    }
+    reduce_row<T, true>(a, sm, gid, tree, r, v_begin, v_count, &part);
+    cluster.sync();  // every slice's partial is complete and visible
+    if (slice == 0) merge_row<T>(a, cluster, &part, gid);
+    cluster.sync();  // nobody rewrites or leaves before the merge has read the partials
   }
 }
 
@@ -337,7 +454,16 @@ cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64
     if (a.n_rows % a.R != 0 || a.n_rows / a.R > 65535) return cudaErrorInvalidValue;
     grid = dim3(a.R, a.n_rows / a.R);
   }
-  if (a.dtype == GTO_BF16)
+  if (a.n_rows <= a.split_below) {
+    // a small batch: kSplit CTAs per row
+    grid.x *= kSplit;
+    if (a.dtype == GTO_BF16)
+      row_reduce_split_kernel<Bf16><<<grid, block, 0, stream>>>(a);
+    else if (a.dtype == GTO_F16)
+      row_reduce_split_kernel<F16><<<grid, block, 0, stream>>>(a);
+    else
+      row_reduce_split_kernel<F32><<<grid, block, 0, stream>>>(a);
+  } else if (a.dtype == GTO_BF16)
     row_reduce_kernel<Bf16><<<grid, block, 0, stream>>>(a);
   else if (a.dtype == GTO_F16)
     row_reduce_kernel<F16><<<grid, block, 0, stream>>>(a);

@@ -37,17 +37,29 @@ def test_config0_all_positions(harness):
     (4104, 4, 3, 17, 16, "f16"),      # fp16 logits (the paper's autocast precision), ragged tail
     (32000, 3, 10, 30, 8, "f16"),
 ])
-def test_small_shapes(harness, V, D, k, g, B, dtype):
+@pytest.mark.parametrize("split", [False, True])
+def test_small_shapes(harness, V, D, k, g, B, dtype, split):
+    """Each shape through the one-CTA-per-row pass and through the cluster-split pass."""
+    from paper_2509_22134_b200 import binding as gto
     w = synth.Workload("t", B=B, V_draft=V, V_target=V, D=D, k=k, g=g, dtype=dtype, seed=V + D)
-    p, data = harness.run_pass(w, DEV)
+    p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_FORCE_ROW_SPLIT if split else 0)
     rep = harness.check_against_oracle(w, p, data, groups=list(range(B // w.m)))
     print(rep)
 
 
-def test_reduced_draft_vocabulary(harness):
+@pytest.mark.parametrize("flags", [0, 16])     # 16 = GTO_FLAG_FORCE_ROW_SPLIT
+def test_reduced_draft_vocabulary(harness, flags):
     w = synth.Workload("t", B=16, V_draft=2048, V_target=8200, D=4, k=5, g=30, seed=77)
-    p, data = harness.run_pass(w, DEV)
+    p, data = harness.run_pass(w, DEV, flags=flags)
     rep = harness.check_against_oracle(w, p, data, groups=[0, 1])
+    print(rep)
+
+
+def test_few_long_rows_take_the_cluster_split_by_themselves(harness):
+    """496 candidate target rows of 256 KB: below the library's own split threshold."""
+    w = synth.Workload("t", B=8, V_draft=32000, V_target=128256, D=4, k=10, g=40, seed=31)
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=[0])
     print(rep)
 
 
@@ -58,6 +70,9 @@ def test_massive_ties_take_the_exact_path(harness):
     data["draft"].zero_()
     data["draft"][:, 1::2, :, :, 100:] = -1.0
     data["target"].zero_()
+    from paper_2509_22134_b200 import binding as gto
+    p, data = harness.run_pass(w, DEV, data=data, flags=gto.GTO_FLAG_FORCE_ROW_SPLIT)
+    harness.check_against_oracle(w, p, data, groups=[0])
     p, data = harness.run_pass(w, DEV, data=data)
     rep = harness.check_against_oracle(w, p, data, groups=[0])
     print(rep)
