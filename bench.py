@@ -42,9 +42,9 @@ NCU_TRAFFIC = {
     # kernel: (source file, sha256 of that file at capture time, bytes per row, V of the capture)
     # from the ncu capture summarised under profiles/ (row pass, workload 2 shapes at B = 64)
     "draft_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                   "fabd0bd90e6442d5051974c8a5dc0790380d78840a67d425e1109255ba330860", (510941696 + 3525120) / 7808, 32000),
+                   "9b80b0d584d978fb10de3ec7706c5b4e528dccfda59000aa34ca2ccb52ccf1a2", (510916864 + 4050432) / 7808, 32000),
     "target_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                    "fabd0bd90e6442d5051974c8a5dc0790380d78840a67d425e1109255ba330860", (429940224 + 3521024) / 1673, 128256),
+                    "9b80b0d584d978fb10de3ec7706c5b4e528dccfda59000aa34ca2ccb52ccf1a2", (429946368 + 3444480) / 1673, 128256),
 }
 
 

@@ -31,7 +31,7 @@ struct gto_ctx {
 };
 
 #ifndef GTO_ROW_SPLIT_ROWS_PER_SM
-#define GTO_ROW_SPLIT_ROWS_PER_SM 6  // up to this many rows per SM, a row is split over a cluster
+#define GTO_ROW_SPLIT_ROWS_PER_SM 10  // up to this many rows per SM, a row is split over a cluster
 #endif
 #ifndef GTO_ROW_GRID_WAVES
 #define GTO_ROW_GRID_WAVES 16  // resident-CTA waves launched for the listed-row pass (measured best of 1..24)
