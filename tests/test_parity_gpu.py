@@ -55,6 +55,31 @@ def test_reduced_draft_vocabulary(harness, flags):
     print(rep)
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_random_shapes(harness, case):
+    """Seeded random shapes inside the compiled limits: vocabulary (ragged tails, fewer vectors
+    than threads), depth, top-k, node budget, group size, logit type, id map, row split."""
+    from paper_2509_22134_b200 import binding as gto
+    rng = np.random.default_rng(1000 + case)
+    dtype = ["bf16", "f16", "f32"][int(rng.integers(3))]
+    per_vec = 4 if dtype == "f32" else 8
+    k = int(rng.integers(1, 12))
+    D = int(rng.integers(1, 9))
+    P = k + (D - 1) * k * k
+    g = int(rng.integers(1, min(P, 128) + 1))
+    Vd = per_vec * int(rng.integers(max(1, -(-k // per_vec)), 1200))
+    reduced = bool(rng.integers(2))
+    Vt = Vd + per_vec * int(rng.integers(1, 600)) if reduced else Vd
+    m = int([1, 2, 4, 8][int(rng.integers(4))])
+    B = m * int(rng.integers(1, 4))
+    w = synth.Workload("rnd", B=B, V_draft=Vd, V_target=Vt, D=D, k=k, g=g, m=m, dtype=dtype,
+                       seed=5000 + case)
+    flags = gto.GTO_FLAG_FORCE_ROW_SPLIT if rng.integers(2) else 0
+    p, data = harness.run_pass(w, DEV, flags=flags)
+    rep = harness.check_against_oracle(w, p, data, groups=list(range(B // m)))
+    print(dict(V=(Vd, Vt), D=D, k=k, g=g, m=m, B=B, dtype=dtype, split=bool(flags)), rep)
+
+
 def test_few_long_rows_take_the_cluster_split_by_themselves(harness):
     """496 candidate target rows of 256 KB: below the library's own split threshold."""
     w = synth.Workload("t", B=8, V_draft=32000, V_target=128256, D=4, k=10, g=40, seed=31)
