@@ -42,7 +42,10 @@ typedef enum {
   GTO_ERR_CUDA = 4,        /* a CUDA runtime call failed                                 */
   GTO_ERR_NONFINITE = 5,   /* device status: a row's log-sum-exp was not finite          */
   GTO_ERR_TIMEOUT = 6,     /* device status: a bounded wait inside a kernel ran out      */
-  GTO_ERR_TOO_LARGE = 7    /* gto_build_tree_noalloc: batch exceeds the fixed scratch    */
+  GTO_ERR_TOO_LARGE = 7,   /* gto_build_tree_noalloc: batch exceeds the fixed scratch    */
+  GTO_ERR_BAD_INDEX = 8    /* device status: an index in a caller's table (d2t, a tree's
+                              rows, tokens or parents, a path's rows) was out of range; the
+                              entry was skipped, results that depend on it are unspecified  */
 } gto_status;
 
 typedef enum { GTO_F32 = 0, GTO_BF16 = 1, GTO_F16 = 2 } gto_dtype;
@@ -226,7 +229,8 @@ gto_status gto_token_loss(gto_ctx* ctx, const void* draft_logits, const void* ta
 gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts);
 
 /* Synchronises `stream`, then reads and clears the device status word:
- * *host_code = GTO_OK, GTO_ERR_NONFINITE or GTO_ERR_TIMEOUT. */
+ * *host_code = GTO_OK, GTO_ERR_NONFINITE, GTO_ERR_BAD_INDEX or GTO_ERR_TIMEOUT.  Kernels check
+ * every index they take from a caller's table before using it as an address. */
 gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code);
 
 /* Number of kernel launches the library has enqueued through this context. */

@@ -118,6 +118,7 @@ const char* gto_status_string(gto_status s) {
     case GTO_ERR_NONFINITE: return "non-finite logit row";
     case GTO_ERR_TIMEOUT: return "bounded device wait ran out";
     case GTO_ERR_TOO_LARGE: return "batch exceeds the fixed scratch of the no-allocation call";
+    case GTO_ERR_BAD_INDEX: return "an index in a caller's table was out of range";
   }
   return "unknown status";
 }
@@ -276,6 +277,7 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
   p.list_count = ctx->list_count;
   p.row_lse_t = out->row_lse_t;
   p.row_argmax_t = out->row_argmax_t;
+  p.status = ctx->status;
   {
     LaunchSpan span(ctx, GTO_K_REWARD_PLAN, s);
     if (gto::launch_reward_plan(p, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
@@ -327,7 +329,9 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
   }
   gto::RewardArgs w{};
   w.B = c.B; w.G = c.G; w.D = c.D; w.k = c.k; w.g = c.g; w.R = ctx->R;
+  w.V_draft = c.V_draft;
   w.V_target = c.V_target;
+  w.status = ctx->status;
   w.dtype = c.logit_dtype;
   w.agg = c.reward_agg;
   w.flags = c.flags;
@@ -381,6 +385,7 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
   a.old_logp = old_logp;
   a.grad = grad;
   a.out = *out;
+  a.status = ctx->status;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   {
     LaunchSpan span(ctx, GTO_K_GROUP_STATS, s);
@@ -447,6 +452,7 @@ gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code) {
       cudaStreamSynchronize(s) != cudaSuccess)
     return GTO_ERR_CUDA;
   *host_code = (word & gto::kStatusTimeout)     ? GTO_ERR_TIMEOUT
+               : (word & gto::kStatusBadIndex)  ? GTO_ERR_BAD_INDEX
                : (word & gto::kStatusNonFinite) ? GTO_ERR_NONFINITE
                                                 : GTO_OK;
   return GTO_OK;

@@ -52,12 +52,14 @@ struct RewardPlanArgs {
   int32_t* list_count;          // out (zeroed by the launcher)
   double* row_lse_t;            // [trees*R] poisoned to NaN for rows not needed
   int32_t* row_argmax_t;        // [trees*R] set to -1 likewise
+  int32_t* status;              // device status word
 };
 cudaError_t launch_reward_plan(const RewardPlanArgs& a, cudaStream_t stream, int64_t* launches);
 
 struct RewardArgs {
-  int B, G, D, k, g, R, V_target, dtype, agg;
+  int B, G, D, k, g, R, V_draft, V_target, dtype, agg;
   uint32_t flags;
+  int32_t* status;
   float eta;
   const void* target;
   const int32_t* d2t;
@@ -76,6 +78,7 @@ struct GradArgs {
   const float* old_logp;
   void* grad;
   gto_grad_stats out;
+  int32_t* status;
 };
 struct TokenLossArgs {
   int B, k, R, V_draft, V_target, dtype;

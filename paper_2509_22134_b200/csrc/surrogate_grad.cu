@@ -48,6 +48,10 @@ __global__ void __launch_bounds__(kStatWarps * 32) group_stats_kernel(GradArgs a
     double R = a.reward.reward[b] - (debias ? a.reward.reward[B + b] : 0.0);
     double A = (R - mean) / (sd + static_cast<double>(a.std_delta));  // Eq. 10
     int l = a.reward.path_len[b];
+    if (l < 0 || l > D) {  // a path has at most D steps
+      atomicOr(a.status, kStatusBadIndex);
+      l = 0;
+    }
     double diff = 0.0, cur = 0.0, old = 0.0;
     for (int j = 0; j < l; ++j) {
       cur += static_cast<double>(a.reward.path_logp[b * D + j]);
@@ -92,6 +96,10 @@ __global__ void __launch_bounds__(kGradThreads) grad_rows_kernel(GradArgs a) {
   }
   const int row = a.reward.path_row[bj];
   const int tok = a.reward.path_token[bj];
+  if (row < 0 || row >= a.R) {  // not a context row: report, write nothing from it
+    if (threadIdx.x == 0) atomicOr(a.status, kStatusBadIndex);
+    return;
+  }
   const float nref =
       -static_cast<float>(a.row_lse[static_cast<size_t>(b) * a.R + row] * 1.4426950408889634);
   const char* in = static_cast<const char*>(a.draft) +

@@ -46,7 +46,12 @@ __global__ void __launch_bounds__(kTokThreads, 8) token_loss_kernel(TokenLossArg
 #pragma unroll
     for (int e = 0; e < E; ++e) {
       const int v = chunk * kChunk + e * 32 + lane;
-      t[e] = v < a.V_draft ? T::load1(zt, __ldg(a.d2t + v)) : -INFINITY;
+      t[e] = -INFINITY;
+      if (v < a.V_draft) {
+        const int id = __ldg(a.d2t + v);
+        if (id >= 0 && id < a.V_target) t[e] = T::load1(zt, id);
+        else atomicOr(a.status, kStatusBadIndex);  // reported; the id counts as probability 0
+      }
     }
   };
   // Without a map: the lane's own 16-byte vector (ids chunk*kChunk + l*E ...).

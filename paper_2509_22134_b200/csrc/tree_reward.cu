@@ -25,6 +25,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) reward_plan_kernel(RewardPl
   __syncwarp();
   for (int n = lane; n < a.g; n += 32) {
     int r = a.node_ctx_row[static_cast<size_t>(tree) * a.g + n];
+    if (r < 0 || r >= a.R) {  // not a row of this tree: report, do not touch memory with it
+      atomicOr(a.status, kStatusBadIndex);
+      continue;
+    }
     atomicOr(&fl[r >> 5], 1u << (r & 31));
   }
   __syncwarp();
@@ -84,15 +88,29 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_reward_kernel(RewardAr
 
   // ---- target probability of every node's token in its context (Eq. 4 factor)
   for (int n = lane; n < g; n += 32) {
-    int ctx = a.tree.node_ctx_row[nb + n];
-    int tok = a.tree.node_token[nb + n];
-    int tt = a.d2t ? a.d2t[tok] : tok;
-    float z = T::load1(tbase, (rb + ctx) * static_cast<size_t>(a.V_target) + tt);
-    double pr = exp(static_cast<double>(z) - a.out.row_lse_t[rb + ctx]);
+    const int ctx = a.tree.node_ctx_row[nb + n];
+    const int tok = a.tree.node_token[nb + n];
+    const int par = a.tree.node_parent[nb + n];
+    const int dep = a.tree.node_depth[nb + n];
+    // every index is checked before it addresses anything
+    bool ok = ctx >= 0 && ctx < R && tok >= 0 && tok < a.V_draft && par >= -1 && par < n &&
+              dep >= 1 && dep <= D;
+    int tt = -1;
+    if (ok) {
+      tt = a.d2t ? a.d2t[tok] : tok;
+      ok = tt >= 0 && tt < a.V_target;
+    }
+    double pr = 0.0;
+    if (ok) {
+      const float z = T::load1(tbase, (rb + ctx) * static_cast<size_t>(a.V_target) + tt);
+      pr = exp(static_cast<double>(z) - a.out.row_lse_t[rb + ctx]);
+    } else {
+      atomicOr(a.status, kStatusBadIndex);
+    }
     sm.p[n] = pr;
-    sm.parent[n] = a.tree.node_parent[nb + n];
-    sm.depth[n] = a.tree.node_depth[nb + n];
-    sm.tok_t[n] = tt;
+    sm.parent[n] = ok ? par : -1;
+    sm.depth[n] = ok ? dep : 1;
+    sm.tok_t[n] = ok ? tt : -1;
     sm.has_child[n] = 0;
   }
   __syncwarp();
@@ -175,6 +193,10 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_reward_kernel(RewardAr
       int slot = a.tree.node_slot[nb + found];
       int depth = sm.depth[found];
       if (slot < 0 || depth >= D) break;
+      if (slot >= k) {  // not a frontier slot: report and stop the walk
+        if (lane == 0) atomicOr(a.status, kStatusBadIndex);
+        break;
+      }
       cur = found;
       row = 1 + (depth - 1) * k + slot;
     }

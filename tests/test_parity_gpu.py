@@ -238,6 +238,61 @@ def test_the_three_calls_can_be_captured_in_a_cuda_graph_and_replayed(harness):
     assert torch.equal(p.grad, p_ref.grad)
 
 
+def test_out_of_range_indices_in_caller_tables_are_reported_not_followed(harness):
+    """Every index a kernel takes from a caller's table (the id map, a tree's rows / tokens /
+    parents, a path's rows and length) is checked before it addresses memory: a bad one sets
+    GTO_ERR_BAD_INDEX in the device status word and is skipped."""
+    from paper_2509_22134_b200.runner import GtoPass
+    BAD = 8
+    w = synth.Workload("t", B=16, V_draft=2048, V_target=8200, D=4, k=5, g=30, seed=77)
+    p_ref, data = harness.run_pass(w, DEV)
+    R = w.R
+
+    def fresh():
+        p = GtoPass(w, DEV)
+        p.build_tree(data["draft"])
+        return p
+
+    # the id map: an id beyond the target vocabulary and a negative one, at tokens the trees use
+    p = fresh()
+    d2t = data["d2t"].clone()
+    used = p.tree["node_token"][0, 0, :2].long()
+    d2t[used[0]] = w.V_target + 1000
+    d2t[used[1]] = -5
+    p.tree_reward(data["target"], d2t)
+    assert p.status() == BAD and p.status() == 0
+    p.token_loss(data["draft"], data["target"], d2t, 1.0)
+    assert p.status() == BAD
+
+    # a tree whose node points at a row, a parent and a token that do not exist
+    p = fresh()
+    p.tree["node_ctx_row"][0, 0, 3] = R + 7
+    p.tree["node_ctx_row"][1, 2, 0] = -2
+    p.tree["node_parent"][0, 1, 4] = w.g + 3
+    p.tree["node_token"][1, 1, 1] = w.V_draft + 9
+    p.tree_reward(data["target"], data["d2t"])
+    assert p.status() == BAD
+
+    # a path with a row outside the tree, and a length beyond the depth
+    p = fresh()
+    p.tree_reward(data["target"], data["d2t"])
+    p.old_logp.copy_(p_ref.old_logp)
+    assert p.status() == 0
+    b = int(torch.nonzero(p.reward["path_len"] > 0)[0])
+    p.reward["path_row"][b, 0] = R + 3
+    p.reward["path_len"][(b + 1) % w.B] = w.D + 5
+    p.surrogate_grad(data["draft"])
+    assert p.status() == BAD
+
+    # the context is fine afterwards: a clean pass reproduces the reference
+    p = fresh()
+    p.tree_reward(data["target"], data["d2t"])
+    p.old_logp.copy_(p_ref.old_logp)
+    p.surrogate_grad(data["draft"])
+    assert p.status() == 0
+    assert torch.equal(p.grad, p_ref.grad) and torch.equal(p.reward["reward"], p_ref.reward["reward"])
+
+
 def test_deterministic_integer_outputs(harness):
     w = synth.WORKLOADS[1].with_B(32)
     p1, data = harness.run_pass(w, DEV)
