@@ -142,8 +142,8 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
         assert _close(gpu["loss"][g0 // m], sur["loss"][0], rtol=REL_TOL, atol=1e-9)
         for j, i in enumerate(idx):
             l = path_len[j]
-            d_i = np.asarray(draft[0, i], dtype=np.float64).reshape(D * k, -1)
-            rows = [d_i[0 if r == 0 else k + r - 1] for r in path_row[j, :l]]
+            d_i = np.asarray(draft[0, i], dtype=np.float64)
+            rows = [d_i[orc.draft_slot_of_row(int(r), k)] for r in path_row[j, :l]]
             lse = [fwd[i]["trees"][0].row_lse[r] for r in path_row[j, :l]]
             want = orc.surrogate_grad_rows(rows, lse, list(path_tok[j, :l]), sur["coeff"][j], D,
                                            draft.shape[-1])

@@ -98,6 +98,12 @@ def context_row(d, j, k):
     return 0 if d == 0 else 1 + (d - 1) * k + j
 
 
+def draft_slot_of_row(r, k):
+    """Inverse of context_row: (d, j) such that the draft tensor [D, k, V] holds context
+    row r at [d, j] (row 0 is the root at [0, 0]; [0, 1:] holds no context)."""
+    return (0, 0) if r == 0 else (1 + (r - 1) // k, (r - 1) % k)
+
+
 def _decision_gap(pool, a, b):
     """Score gap between two candidates that a ranking decision separates.  Two
     children of one parent with the same logit tie exactly on every implementation
@@ -413,8 +419,8 @@ def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, ag
     grad = np.zeros((m, D, V))
     for i, f in enumerate(fwd):
         l = path_len[i]
-        d_i = np.asarray(draft_g[0, i], dtype=np.float64).reshape(D * k, V)
-        rows = [d_i[0 if r == 0 else k + r - 1] for r in path_row[i, :l]]
+        d_i = np.asarray(draft_g[0, i], dtype=np.float64)          # [D, k, V] of the current draft
+        rows = [d_i[draft_slot_of_row(int(r), k)] for r in path_row[i, :l]]
         lse = [f["trees"][0].row_lse[r] for r in path_row[i, :l]]
         grad[i] = surrogate_grad_rows(rows, lse, list(path_tok[i, :l]), sur["coeff"][i], D, V)
     return dict(fwd=fwd, R=R, A=A, path_len=path_len, path_logp=path_logp, path_row=path_row,

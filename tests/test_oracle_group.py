@@ -39,6 +39,11 @@ def test_advantages_special_cases():
     assert np.allclose(An, A)
 
 
+# factor on the summed group losses for each seed of the autograd pin: 1, and the
+# omega / K = 0.5 / 16 a trainer passes with the settings of App. B
+GRAD_SCALES = [1.0, 0.5 / 16, 3.0, 0.5 / 16]
+
+
 def torch_loss(z, rows_tok, old, adv, m, eps):
     """Eq. 11-12 written with torch ops on leaf logits z[b][j]; autograd differentiates."""
     total = 0.0
@@ -65,12 +70,13 @@ def test_gradient_matches_autograd_and_finite_differences(seed):
         for j in range(lens[b]):
             path_logp[b, j] = rows[b][j][toks[b][j]] - lse[b][j]
     old = path_logp + rng.normal(size=(B, D)) * 0.6       # some ratios leave the clip range
-    sur = orc.clipped_surrogate(path_logp, old, lens, adv, m, eps=eps, grad_scale=1.0)
+    scale = GRAD_SCALES[seed]
+    sur = orc.clipped_surrogate(path_logp, old, lens, adv, m, eps=eps, grad_scale=scale)
     assert (~sur["active"]).any() and sur["active"].any()
     z = [[torch.tensor(r, dtype=torch.float64, requires_grad=True) for r in rs] for rs in rows]
     loss = torch_loss(z, toks, old, adv, m, eps)
     assert float(loss.detach()) == pytest.approx(float(sur["loss"].sum()), rel=1e-12)
-    loss.backward()
+    (scale * loss).backward()           # the gradient is that of grad_scale * sum_k loss_k
     for b in range(B):
         got = orc.surrogate_grad_rows(rows[b], lse[b], toks[b], sur["coeff"][b], D, V)
         for j in range(D):
@@ -93,7 +99,7 @@ def test_gradient_matches_autograd_and_finite_differences(seed):
                 pl = path_logp.copy()
                 for jj in range(lens[b]):
                     pl[b, jj] = rr[jj][toks[b][jj]] - np.log(np.sum(np.exp(rr[jj])))
-                return orc.clipped_surrogate(pl, old, lens, adv, m, eps=eps)["loss"].sum()
+                return scale * orc.clipped_surrogate(pl, old, lens, adv, m, eps=eps)["loss"].sum()
             fd = (total(h) - total(-h)) / (2 * h)
             got = orc.surrogate_grad_rows(rows[b], lse[b], toks[b], sur["coeff"][b], D, V)[j, v]
             assert abs(fd - got) < 1e-7

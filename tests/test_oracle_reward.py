@@ -196,6 +196,64 @@ def test_walk_stops_at_unexpanded_node_and_on_mismatch():
     assert orc.longest_accepted(tree, target)["nodes"] == []
 
 
+def _worked_tree_with_id_map():
+    """D = 3, k = 2, draft vocabulary 4 mapped into a target vocabulary of 9 by (1, 4, 6, 8).
+    Worked by hand: the root proposes tokens 0 and 1 (slots 0, 1); under token 0 the draft
+    proposes 2 and 3, which outrank both children of token 1 and become slots 0 and 1 of
+    depth 2 (context rows 3 and 4); the six best candidates are the pool indices
+    0, 1, 2, 3, 6 (path 0-2-0) and 8 (path 0-3-1), listed in that order."""
+    D, k = 3, 2
+    d2t = np.array([1, 4, 6, 8])
+    draft = np.zeros((D, k, 4))
+    draft[0, 0] = [5, 4, 0, 0]
+    draft[0, 1] = np.nan                       # no context lives here
+    draft[1, 0] = [0, 0, 5, 4]
+    draft[1, 1] = [-9, -9, -9, -9.5]
+    draft[2, 0] = [1, 0, 0, 0]
+    draft[2, 1] = [0, 3, 0, 0]
+    tree = orc.build_tree(draft, D, k, 6)
+    assert list(tree.pool) == [0, 1, 2, 3, 6, 8]
+    assert list(tree.token) == [0, 1, 2, 3, 0, 1]
+    return tree, d2t
+
+
+def test_walk_compares_the_greedy_target_id_with_the_mapped_draft_id():
+    """Sec. 3.2 / App. A case (b) with a reduced draft vocabulary: the target's greedy token
+    is a TARGET id, a child matches when the image of its draft id under the map equals it.
+    The greedy ids are chosen so that a walk that compared raw draft ids would go elsewhere:
+    at the root the target picks id 1 = map(0), and a child with draft id 1 exists too."""
+    tree, d2t = _worked_tree_with_id_map()
+    target = np.full((5, 9), -50.0)
+    target[0, 1] = 50.0          # map(0): accept token 0 (list position 0)
+    target[1, 8] = 50.0          # map(3) in the context of token 0: accept 0-3 (position 3, slot 1)
+    target[4, 4] = 50.0          # map(1) in context row 4 = slot 1 of depth 2: accept 0-3-1 (position 5)
+    target[2, 4] = 50.0          # rows the walk must not consult
+    target[3, 1] = 50.0
+    path = orc.longest_accepted(tree, target, d2t)
+    assert path["nodes"] == [0, 3, 5]
+    assert path["rows"] == [0, 1, 4]
+    assert path["tokens"] == [0, 3, 1]           # draft ids, not target ids
+    assert path["logp"] == pytest.approx([5 - np.log(np.exp(5) + np.exp(4) + 2),
+                                          4 - np.log(np.exp(5) + np.exp(4) + 2),
+                                          3 - np.log(np.exp(3) + 3)], abs=1e-12)
+    # the identity map on a shared vocabulary is the same thing as no map
+    same = orc.longest_accepted(tree, target[:, :4] + 0.0, np.arange(4))
+    assert same == orc.longest_accepted(tree, target[:, :4] + 0.0, None)
+
+
+def test_greedy_target_token_outside_the_image_of_the_map_accepts_nothing():
+    """A target id no draft id maps to cannot be drafted: the walk stops, also when a child
+    happens to carry that number as its draft id."""
+    tree, d2t = _worked_tree_with_id_map()
+    target = np.full((5, 9), -50.0)
+    target[0, 0] = 50.0          # target id 0 is not in (1, 4, 6, 8); draft id 0 is a child of the root
+    assert orc.longest_accepted(tree, target, d2t)["nodes"] == []
+    target[0] = -50.0
+    target[0, 1] = 50.0          # accept token 0 ...
+    target[1, 2] = 50.0          # ... then target id 2: unmapped, while draft id 2 is a child there
+    assert orc.longest_accepted(tree, target, d2t)["nodes"] == [0]
+
+
 def test_all_nodes_variant_sums_over_every_root_to_node_sequence():
     """Independent restatement: walk every node's path with explicit products."""
     draft, target, tree = tiny_case(11, V=6, D=4, k=3, g=12)

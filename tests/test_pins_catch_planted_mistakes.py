@@ -8,6 +8,7 @@ import pytest
 from oracle import gto_oracle as orc
 
 import test_oracle_group as tg
+import test_oracle_pass as tp
 import test_oracle_reward as tr
 import test_oracle_rows as trow
 import test_oracle_token_loss as tt
@@ -182,3 +183,39 @@ def test_tree_scored_by_the_edge_probability_instead_of_the_path(monkeypatch):
     monkeypatch.setattr(orc, "build_tree", build)
     assert fails(ttree.test_fig1_greedy_leaf_is_pruned_by_a_better_sibling_path) or \
         fails(ttree.test_tree_invariants_default_shape, 0)
+
+
+def test_walk_that_ignores_the_id_map(monkeypatch):
+    """Sec. 3.2 with a reduced draft vocabulary: comparing the greedy target id with the raw
+    draft id instead of its image under the map."""
+    real = orc.longest_accepted
+    monkeypatch.setattr(orc, "longest_accepted", lambda tree, target, d2t=None: real(tree, target, None))
+    assert fails(tr.test_walk_compares_the_greedy_target_id_with_the_mapped_draft_id)
+    assert fails(tr.test_greedy_target_token_outside_the_image_of_the_map_accepts_nothing)
+
+
+def test_surrogate_that_drops_the_gradient_scale(monkeypatch):
+    real = orc.clipped_surrogate
+    monkeypatch.setattr(orc, "clipped_surrogate",
+                        lambda path_logp, old_logp, path_len, adv, m, eps=0.2, grad_scale=1.0:
+                        real(path_logp, old_logp, path_len, adv, m, eps, 1.0))
+    assert fails(tg.test_gradient_matches_autograd_and_finite_differences, 1)
+    assert fails(tp.test_hand_worked_group_rows_tokens_and_advantages_land_where_they_belong)
+
+
+def test_pass_that_reads_the_gradient_rows_from_the_wrong_draft_row(monkeypatch):
+    """The draft tensor keeps k - 1 unused rows after the root: an index that forgets them."""
+    monkeypatch.setattr(orc, "draft_slot_of_row", lambda r, k: (r // k, r % k))
+    assert fails(tp.test_hand_worked_group_rows_tokens_and_advantages_land_where_they_belong)
+    assert fails(tp.test_whole_pass_gradient_by_finite_differences_over_every_draft_logit)
+
+
+def test_pass_that_hands_the_advantages_to_the_wrong_positions(monkeypatch):
+    real = orc.group_advantages
+
+    def mutant(rc, rr, m, delta=1e-6, unbiased=False, debias=True):
+        R, A = real(rc, rr, m, delta, unbiased, debias)
+        return R, A[::-1].copy()
+    monkeypatch.setattr(orc, "group_advantages", mutant)
+    # (finite differences cannot see this one: loss and gradient would use the same wrong values)
+    assert fails(tp.test_hand_worked_group_rows_tokens_and_advantages_land_where_they_belong)
