@@ -8,6 +8,18 @@ With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs
 number of its own positions (weak scaling); positions are independent, so no collective is
 on the data path - only the timing barrier and the max-over-ranks reduction.
 
+Started directly with --gpus N > 1 (no WORLD_SIZE in the environment) it starts the N ranks
+itself under torch.distributed.run.
+
+Timed regions of the GPU arm, in order: (1) the headline: K steps, nothing but the three
+calls; (2) the same K steps with every kernel launch bracketed by CUDA events, for the
+per-kernel split and the roofline; (3) a sustained region of at least a second of
+back-to-back steps, with the SM clock sampled, to show where the pass settles under the
+board power limit; (4) the end-to-end leg with the logits in pinned host memory.  At N = 1
+the oracle then runs on every host core over groups drawn from the same batch: its
+throughput is the CPU baseline, and its results are compared with the library's for those
+groups (the `parity` counts).
+
 Prints ONE JSON line on rank 0.  `--impl reference` times the fp64 CPU oracle instead (on a
 bounded sample per step), on rank 0 only.
 """
@@ -16,8 +28,11 @@ from __future__ import annotations
 import argparse
 import hashlib
 import json
+import math
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -34,6 +49,8 @@ UNIT = "positions/s"
 HBM_FALLBACK_GBS = 6650.0
 REFERENCE_BUDGET_S = 150.0  # the oracle arm stops taking new steps after this much wall time
 E2E_POSITIONS = 64          # positions per end-to-end step (host buffers of ~2.6 GB at workload 2)
+SUSTAINED_SECONDS = 1.2     # length of the back-to-back region
+COOLDOWN_SECONDS = 1.0      # idle time before the per-kernel region
 
 # DRAM traffic per processed row of the dominant kernels, from one ncu capture each
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch / rows in the launch).  An
@@ -71,7 +88,7 @@ class ClockSampler:
 
     def __init__(self, device_index: int, period_s: float = 0.01):
         self.period = period_s
-        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.samples, self.stamps, self.reasons, self.max_mhz = [], [], set(), None
         self._stop = threading.Event()
         self._thread = None
         self._h = None
@@ -92,6 +109,7 @@ class ClockSampler:
         while not self._stop.is_set():
             try:
                 self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                self.stamps.append(time.perf_counter())
                 mask = int(get_reasons(self._h))
                 for bit, name in self._REASONS.items():
                     if mask & bit:
@@ -118,86 +136,165 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------ oracle legs
-def _oracle_group_fn(w):
-    """Returns f(draft_g, target_g, d2t, b0) running the oracle's whole pass on one group."""
+# Everything between here and workload_config is the CPU-baseline / reference leg: the only
+# part of this file that runs the oracle.  The functions named *_task run in worker processes.
+def _old_logp_fn(w, with_positions):
+    from paper_2509_22134_b200 import synth
+
+    def at(path_logp, path_row, path_token, path_len, first_of):
+        out = np.zeros_like(path_logp)
+        for i in range(path_logp.shape[0]):
+            out[i] = synth.old_logp_from_path(w, path_logp[i:i + 1], path_row[i:i + 1],
+                                              path_token[i:i + 1], path_len[i:i + 1], b0=first_of(i))[0]
+        return out
+    if with_positions:
+        return lambda pl, pr, pt, ln, positions: at(pl, pr, pt, ln, lambda i: positions[i])
+    return lambda b0: (lambda pl, pr, pt, ln: at(pl, pr, pt, ln, lambda i: b0 + i))
+
+
+def oracle_group_task(w, draft, draft_tag, target, target_tag, d2t, b0, gpu=None):
+    """The oracle's whole pass on one group of m positions (first absolute position b0)."""
     from oracle import gto_oracle as orc
-    from paper_2509_22134_b200 import synth
-
-    def run(draft_g, target_g, d2t, b0):
-        def old_fn(path_logp, path_row, path_token, path_len):
-            out = np.zeros_like(path_logp)
-            for i in range(path_logp.shape[0]):
-                out[i] = synth.old_logp_from_path(w, path_logp[i:i + 1], path_row[i:i + 1],
-                                                  path_token[i:i + 1], path_len[i:i + 1], b0=b0 + i)[0]
-            return out
-        return orc.group_pass(draft_g, target_g, w.D, w.k, w.g, w.m, old_fn, d2t, w.eta,
-                              delta=w.std_delta, eps=w.clip_eps, grad_scale=w.grad_scale)
-    return run
+    from oracle import parallel as opar
+    out = orc.group_pass(opar.decode_logits(draft, draft_tag), opar.decode_logits(target, target_tag),
+                         w.D, w.k, w.g, w.m, _old_logp_fn(w, False)(b0), d2t, w.eta,
+                         delta=w.std_delta, eps=w.clip_eps, grad_scale=w.grad_scale)
+    return float(out["sur"]["loss"][0])
 
 
-def _sample_groups(w, n_groups, device):
-    """Synthetic logits of the first n_groups groups, as host fp32 arrays (exact values)."""
-    from paper_2509_22134_b200 import synth
-    data = synth.generate(w.with_B(n_groups * w.m), device)
-    draft = data["draft"].float().cpu().numpy()
-    target = data["target"].float().cpu().numpy()
+def oracle_check_task(w, draft, draft_tag, target, target_tag, d2t, b0, gpu):
+    """The library's outputs for one group against the oracle (tolerances of oracle/check.py)."""
+    from oracle import check as ocheck
+    from oracle import parallel as opar
+
+    class Cfg:
+        pass
+    cfg = Cfg()
+    for name in ("B", "G", "D", "k", "g", "m", "eta", "clip_eps", "std_delta", "grad_scale"):
+        setattr(cfg, name, getattr(w, name))
+    try:
+        return ocheck.check_positions(cfg, opar.decode_logits(draft, draft_tag),
+                                      opar.decode_logits(target, target_tag), d2t, gpu,
+                                      _old_logp_fn(w, True), list(range(b0, b0 + w.m)))
+    except AssertionError as e:
+        return {"positions": w.m, "failed": 1, "failure": str(e)[:300]}
+
+
+def _group_payload(w, data, gidx, first_position, p=None):
+    """Logits (and, with p, the library's outputs) of group gidx of the batch in `data`."""
+    from oracle import parallel as opar
+    sl = slice(gidx * w.m, (gidx + 1) * w.m)
+    draft, dtag = opar.encode_logits(data["draft"][:, sl])
+    target, ttag = opar.encode_logits(data["target"][:, sl])
     d2t = None if data["d2t"] is None else data["d2t"].cpu().numpy().astype(np.int64)
-    return draft, target, d2t
+    gpu = None
+    if p is not None:
+        gpu = {}
+        for name, t in p.tree.items():
+            gpu[name] = t[:, sl].cpu().numpy()
+        for name, t in p.reward.items():
+            gpu[name] = (t[sl] if name.startswith("path_") else t[:, sl]).cpu().numpy()
+        for name, t in p.stats.items():
+            gpu[name] = (t[gidx:gidx + 1] if name == "loss" else t[sl]).cpu().numpy()
+        gpu["grad"] = p.grad[sl].float().cpu().numpy().astype(np.float64)
+        # rows that carry no gradient are the caller's with GTO_FLAG_GRAD_LIVE_ROWS: the method's value there is 0
+        j = np.arange(w.D)[None, :]
+        dead = ~((j < gpu["path_len"][:, None]) & (gpu["coeff"][:, None] != 0))
+        gpu["grad"][dead] = 0.0
+    return dict(w=w, draft=draft, draft_tag=dtag, target=target, target_tag=ttag, d2t=d2t,
+                b0=first_position + gidx * w.m, gpu=gpu)
 
 
-def cpu_baseline(w, device, budget_s=12.0, max_groups=4):
-    """Oracle throughput on whole groups of the workload until ~budget_s of CPU work."""
-    run = _oracle_group_fn(w)
-    draft, target, d2t = _sample_groups(w, max_groups, device)
+def _host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline_and_parity(w, data, p, first_position, budget_s=25.0):
+    """The oracle on every host core over whole groups drawn (seeded) from the benchmarked
+    batch: one group per core, a second wave if the first took under half the budget.
+    Returns (cpu_baseline, parity): the throughput of the oracle's pass, and the comparison
+    of the library's outputs for the same groups."""
+    from oracle.parallel import OracleWorkers
+    cores = _host_cores()
+    n_groups = w.B // w.m
+    rng = np.random.default_rng(w.seed % (1 << 32))
+    order = [0] + [int(x) for x in rng.permutation(np.arange(1, n_groups))]
     torch.set_num_threads(1)
-    done, t0 = 0, time.perf_counter()
-    for gidx in range(max_groups):
-        sl = slice(gidx * w.m, (gidx + 1) * w.m)
-        run(draft[:, sl], target[:, sl], d2t, gidx * w.m)
-        done += w.m
-        if time.perf_counter() - t0 >= budget_s:
-            break
-    dt = time.perf_counter() - t0
-    return {"value": done / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"first {done} positions ({done // w.m} groups of m={w.m}) of the workload, "
-                      f"{dt:.1f} s, fp64 numpy, one host thread of {os.cpu_count()}"}
+    done, wall, cpu_s, reps = [], 0.0, 0.0, []
+    with OracleWorkers(min(cores, n_groups)) as pool:
+        for wave in range(2):
+            groups = order[len(done):len(done) + pool.n]
+            if not groups:
+                break
+            for i, gidx in enumerate(groups):
+                pool.put(i, _group_payload(w, data, gidx, first_position, p))
+            keys = list(range(len(groups)))
+            _, dt, per = pool.call("bench", "oracle_group_task", keys, drop=False)
+            wall += dt
+            cpu_s += sum(per.values())
+            res, _, _ = pool.call("bench", "oracle_check_task", keys)
+            reps += [res[i] for i in keys]
+            done += groups
+            if wall > budget_s / 2:
+                break
+    n_pos = len(done) * w.m
+    base = {"value": n_pos / wall, "unit": UNIT, "cores": min(cores, n_groups), "kind": "oracle",
+            "per_core": n_pos / cpu_s,
+            "sample": f"{n_pos} positions = {len(done)} whole groups of m={w.m} drawn over the batch "
+                      f"(group 0 and a seeded permutation), one group per worker process, "
+                      f"{wall:.1f} s wall, fp64 numpy, one thread per process, {cores} host cores"}
+    parity = {"groups_checked": len(done), "positions_checked": n_pos, "groups": sorted(done),
+              "failed_groups": sum(r.get("failed", 0) for r in reps),
+              "near_tie_trees": sum(r.get("near_tie_trees", 0) for r in reps),
+              "clip_edge": sum(r.get("clip_edge", 0) for r in reps),
+              "ill_conditioned_groups": sum(r.get("ill_conditioned_groups", 0) for r in reps)}
+    for key in ("max_lse_err", "max_score_err", "max_reward_rel", "max_adv_err", "max_grad_err"):
+        parity[key] = max((r.get(key, 0.0) for r in reps), default=0.0)
+    fails = [r["failure"] for r in reps if r.get("failed")]
+    if fails:
+        parity["first_failure"] = fails[0]
+    return base, parity
 
 
 def run_reference(args, w, rank, world):
-    """The oracle as the reference arm: one group of m positions per step, rank 0 only."""
+    """The oracle as the reference arm, rank 0 only: every step runs one whole group of m
+    positions of the workload on each host core (the same groups every step)."""
     if rank != 0:
         return
+    from oracle.parallel import OracleWorkers
+    from paper_2509_22134_b200 import synth
     device = "cuda:0" if torch.cuda.is_available() else "cpu"
-    run = _oracle_group_fn(w)
-    n_groups = 2
-    draft, target, d2t = _sample_groups(w, n_groups, device)
+    cores = _host_cores()
+    n_workers = max(1, min(cores, w.B // w.m))
+    data = synth.generate(w.with_B(n_workers * w.m), device)
     torch.set_num_threads(1)
-
-    def step(i):
-        gidx = i % n_groups
-        sl = slice(gidx * w.m, (gidx + 1) * w.m)
-        run(draft[:, sl], target[:, sl], d2t, gidx * w.m)
-
     wall0 = time.perf_counter()
-    for i in range(args.warmup):
-        step(i)
-    t0 = time.perf_counter()
-    done = 0
-    for i in range(args.steps):
-        step(i)
-        done += 1
-        if time.perf_counter() - wall0 > REFERENCE_BUDGET_S:   # keep the run to a few minutes
-            break
-    dt = time.perf_counter() - t0
-    value = done * w.m / dt
-    sample = (f"each step = one group of m={w.m} positions of the workload (groups 0..{n_groups - 1} "
-              f"in turn), fp64 numpy, one host thread of {os.cpu_count()}")
+    with OracleWorkers(n_workers) as pool:
+        for i in range(n_workers):
+            pool.put(i, _group_payload(w, data, i, 0))
+        keys = list(range(n_workers))
+        del data
+        times = []
+        for i in range(args.warmup + args.steps):
+            _, dt, _ = pool.call("bench", "oracle_group_task", keys, drop=False)
+            if i >= args.warmup:
+                times.append(dt)
+            if times and time.perf_counter() - wall0 > REFERENCE_BUDGET_S:   # keep the run to a few minutes
+                break
+    done, dt = len(times), sum(times)
+    value = done * n_workers * w.m / dt
+    sample = (f"each step = {n_workers} whole groups of m={w.m} positions of the workload (groups "
+              f"0..{n_workers - 1}, the same every step), one group per worker process, fp64 numpy, one "
+              f"thread per process, {cores} host cores")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": done, "steps_requested": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * dt / max(done, 1),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": workload_config(w, args.gpus),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": n_workers, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -242,6 +339,46 @@ def algorithmic_bytes(w, p):
     }
 
 
+def timed_steps(p, data, n, stream, barrier, clocks=None):
+    """n back-to-back steps bracketed by barrier + synchronize; returns (total ms, per-step ms,
+    host time stamps of the region's start and end)."""
+    ev0 = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.perf_counter()
+    ev0.record(stream)
+    marks = []
+    for _ in range(n):
+        p.step(data["draft"], data["target"], data["d2t"])
+        marks.append(torch.cuda.Event(enable_timing=True))
+        marks[-1].record(stream)
+    barrier()
+    t1 = time.perf_counter()
+    per_step = [a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks)]
+    return ev0.elapsed_time(marks[-1]), per_step, (t0, t1)
+
+
+def by_clock(per_step, span, clocks, step_bytes):
+    """Steps binned by the SM clock sampled while they ran (the device runs the queued steps
+    back to back, so a sample's place between the region's host time stamps is its place in
+    the step sequence).  Returns [{sm_mhz (bin centre), steps, ms_per_step, gbs}], fastest first."""
+    if not clocks.samples:
+        return []
+    t0, t1 = span
+    ends = np.cumsum(per_step) / max(sum(per_step), 1e-9)
+    bins = {}
+    for mhz, ts in zip(clocks.samples, clocks.stamps):
+        if not (t0 <= ts <= t1):
+            continue
+        i = min(int(np.searchsorted(ends, (ts - t0) / (t1 - t0))), len(per_step) - 1)
+        bins.setdefault(int(round(mhz / 50.0)) * 50, set()).add(i)
+    out = []
+    for mhz, steps in sorted(bins.items(), reverse=True):
+        ms = statistics.mean(per_step[i] for i in steps)
+        out.append({"sm_mhz": mhz, "steps": len(steps), "ms_per_step": ms,
+                    "gbs": step_bytes / (ms * 1e-3) / 1e9})
+    return out
+
+
 def run_gpu(args, w, rank, world, local_rank):
     from paper_2509_22134_b200 import binding as gto
     from paper_2509_22134_b200 import synth
@@ -252,11 +389,13 @@ def run_gpu(args, w, rank, world, local_rank):
     b0 = shard_first_position(rank, w.B)
     data = synth.generate(w, dev, b0=b0)
     p = GtoPass(w, dev, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS)
+    p.grad.zero_()   # rows without a gradient are the caller's under GTO_FLAG_GRAD_LIVE_ROWS
     # the old-policy log-probabilities are an input of the gradient call: fix them once
     p.build_tree(data["draft"])
     p.tree_reward(data["target"], data["d2t"])
     p.set_old_logp_from_path(b0=b0)
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         p.step(data["draft"], data["target"], data["d2t"])
     assert p.status() == 0
 
@@ -266,24 +405,30 @@ def run_gpu(args, w, rank, world, local_rank):
         torch.cuda.synchronize(dev)
 
     stream = torch.cuda.current_stream(dev)
-    ev0 = torch.cuda.Event(enable_timing=True)
-    gto.gto_kernel_timing(p.ctx, True)
+    # ---- (1) the headline region: K steps, the three calls and nothing else
     launches0 = p.launches()
     with ClockSampler(local_rank) as clocks:
-        barrier()
-        ev0.record(stream)
-        marks = []
-        for _ in range(args.steps):
-            p.step(data["draft"], data["target"], data["d2t"])
-            marks.append(torch.cuda.Event(enable_timing=True))
-            marks[-1].record(stream)
-        ev1 = marks[-1]
-        barrier()
-    ms = ev0.elapsed_time(ev1)
-    per_step = [a.elapsed_time(b) for a, b in zip([ev0] + marks[:-1], marks)]
+        ms, per_step, _ = timed_steps(p, data, args.steps, stream, barrier)
+    launches = p.launches() - launches0
+    # ---- (2) the same with every launch bracketed by events: the per-kernel split.  The board
+    #      idles for a moment first so that this region starts from the same power state as
+    #      the first one (a few hundred ms of back-to-back steps already lower the clock).
+    time.sleep(COOLDOWN_SECONDS)
+    gto.gto_kernel_timing(p.ctx, True)
+    for _ in range(3):
+        p.step(data["draft"], data["target"], data["d2t"])
+    gto.gto_kernel_times(p.ctx)
+    with ClockSampler(local_rank) as split_clocks:
+        ms_events, _, _ = timed_steps(p, data, args.steps, stream, barrier)
     ktimes = gto.gto_kernel_times(p.ctx)
     gto.gto_kernel_timing(p.ctx, False)
-    launches = p.launches() - launches0
+    # ---- (3) sustained: at least SUSTAINED_SECONDS of back-to-back steps, clocks sampled
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(args.steps, int(math.ceil(SUSTAINED_SECONDS * 1e3 / (ms / args.steps))))
+        with ClockSampler(local_rank) as sus_clocks:
+            sus_ms, sus_steps, sus_span = timed_steps(p, data, n_sus, stream, barrier)
+        sustained = (n_sus, sus_ms, sus_steps, sus_span, sus_clocks)
     assert p.status() == 0
 
     # ---- next-row kernel, timed on its own (not part of the step): token-level loss
@@ -300,15 +445,16 @@ def run_gpu(args, w, rank, world, local_rank):
         tok_bytes = w.B * 3 * w.V_draft * w.elem_bytes   # draft row, mapped target logits, gradient row
         extras["token_loss"] = {"ms": tot / cnt, "algorithmic_bytes": tok_bytes,
                                 "gbs": tok_bytes / (tot / cnt * 1e-3) / 1e9,
-                                "note": "Eq. 13 on the B root rows; the id-map gather touches "
-                                        "nearly every 32-byte sector of the target row"}
+                                "note": "Eq. 13 on the B root rows, timed alone (not part of the step)"}
 
-    # ---- end to end: host buffers, copies inside the timed region
+    # ---- (4) end to end: host buffers, copies inside the timed region
     e2e = run_e2e(args, w, dev, b0, world) if not args.no_e2e else None
     if e2e is None:
-        e2e = {"ms": float("nan"), "positions": 0, "h2d": 0, "d2h": 0, "positions_per_step": 0, "steps": 0}
+        e2e = {"ms": float("nan"), "positions": 0, "h2d": 0, "d2h": 0, "positions_per_step": 0, "steps": 0,
+               "pinned_h2d_gbs": None}
 
-    ms, e2e_ms = max_over_ranks([ms, e2e["ms"]], world, dev)
+    sus_ms_all = sustained[1] if sustained else float("nan")
+    ms, ms_events, e2e_ms, sus_ms_all = max_over_ranks([ms, ms_events, e2e["ms"], sus_ms_all], world, dev)
     if rank != 0:
         return
 
@@ -334,6 +480,10 @@ def run_gpu(args, w, rank, world, local_rank):
                 "unit": "GB/s", "frac": kern[top]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": traffic,
                 "algorithmic_bytes_per_launch": alg[top],
+                "timed_in": f"a second region of {args.steps} steps with every launch bracketed by CUDA "
+                            f"events ({ms_events / args.steps:.4f} ms per step there), after "
+                            f"{COOLDOWN_SECONDS} s of idling",
+                "clocks": split_clocks.summary(),
                 "pass": {"algorithmic_bytes_per_step": step_bytes,
                          "achieved": step_bytes / step_s / 1e9,
                          "frac": step_bytes / step_s / 1e9 / peak,
@@ -341,20 +491,31 @@ def run_gpu(args, w, rank, world, local_rank):
                 "kernels": kern,
                 "counts": {k: alg[k] for k in ("needed_target_rows", "path_rows", "live_grad_rows")}}
     line = {"metric": METRIC, "value": world * w.B * args.steps / (ms * 1e-3), "unit": UNIT,
-            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+            "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms / args.steps, "ms_per_step_median": statistics.median(per_step),
             "ms_per_step_min": min(per_step), "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "vs_baseline": None, "dtype": "f32", "storage_dtype": w.dtype, "data": "synthetic",
             "config": workload_config(w, world),
             "clocks": clocks.summary(),
             "e2e": {"value": world * e2e["positions"] / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                    "positions_per_step": e2e["positions_per_step"], "steps": e2e["steps"]},
+                    "positions_per_step": e2e["positions_per_step"], "steps": e2e["steps"],
+                    "pinned_h2d_gbs": e2e["pinned_h2d_gbs"]},
             "gpu_launches": launches,
             "roofline": roofline,
             "extras": extras}
+    if sustained:
+        n_sus, _, sus_steps, sus_span, sus_clocks = sustained
+        sus_s = sus_ms_all * 1e-3 / n_sus
+        cs = sus_clocks.summary()
+        line["sustained"] = {"steps": n_sus, "seconds": sus_ms_all * 1e-3, "ms_per_step": sus_ms_all / n_sus,
+                             "value": world * w.B / sus_s, "gbs": step_bytes / sus_s / 1e9,
+                             "frac_of_measured": step_bytes / sus_s / 1e9 / peak,
+                             "frac_of_8000_nominal": step_bytes / sus_s / 1e9 / 8000.0,
+                             "sm_mhz_median": cs["sm_mhz"], "reasons": cs["reasons"],
+                             "by_clock": by_clock(sus_steps, sus_span, sus_clocks, step_bytes)}
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(w, dev)
+        line["cpu_baseline"], line["parity"] = cpu_baseline_and_parity(w, data, p, b0)
     print(json.dumps(line), flush=True)
 
 
@@ -401,6 +562,13 @@ def run_e2e(args, w, dev, b0, world):
     for _ in range(3):
         step()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # the bus itself: one plain copy of the pinned draft buffer, for a ceiling beside the figure
+    torch.cuda.synchronize(dev)
+    ev0.record()
+    data["draft"].copy_(host["draft"], non_blocking=True)
+    ev1.record()
+    torch.cuda.synchronize(dev)
+    pinned_gbs = host["draft"].numel() * host["draft"].element_size() / (ev0.elapsed_time(ev1) * 1e-3) / 1e9
     if world > 1:
         torch.distributed.barrier()
     torch.cuda.synchronize(dev)
@@ -416,7 +584,18 @@ def run_e2e(args, w, dev, b0, world):
     h2d = h2d_fixed + rows[0] * row_bytes   # + the row list read back (counted in d2h)
     d2h += 4 * (we.G * we.B * we.R + 1)
     return {"ms": ms, "positions": we.B * steps, "h2d": h2d, "d2h": d2h,
-            "positions_per_step": we.B, "steps": steps}
+            "positions_per_step": we.B, "steps": steps, "pinned_h2d_gbs": pinned_gbs}
+
+
+def spawn_ranks(n: int) -> int:
+    """Started without a launcher: run this same command line as n ranks on this node (one per
+    GPU, rank r on GPU r) under torch.distributed.run, and return its exit code."""
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd).returncode
 
 
 def main():
@@ -429,6 +608,7 @@ def main():
     ap.add_argument("--positions", type=int, default=None, help="override B (a multiple of m)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the back-to-back region (profiling runs)")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 3 if args.impl == "reference" else 50
@@ -447,8 +627,12 @@ def main():
     if args.impl == "reference":
         run_reference(args, w, rank, world)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device (the GTO pass has no CPU path)")
+        raise SystemExit(f"bench.py: no CUDA device on rank {rank} (the GTO pass has no CPU path)")
+    if torch.cuda.device_count() <= local_rank:
+        raise SystemExit(f"bench.py: rank {rank} wants GPU {local_rank}, the node has {torch.cuda.device_count()}")
     if world > 1:
         torch.cuda.set_device(local_rank)
         torch.distributed.init_process_group("nccl", device_id=torch.device("cuda", local_rank))

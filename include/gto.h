@@ -215,16 +215,35 @@ typedef struct {
  * out->loss[b] and grad_root[b,:] = weight * (p_M - p_T), the derivative of weight * H with
  * respect to the draft logits of that row ([B, V_draft], logit dtype, every entry written);
  * a trainer passes weight = 1 / (number of supervised positions).  Needs tree->row_lse from
- * gto_build_tree on the same draft logits. */
+ * gto_build_tree on the same draft logits.  An increasing d2t (a vocabulary subset listed in
+ * id order) is streamed at memory bandwidth; any other injective map is gathered, slower. */
 gto_status gto_token_loss(gto_ctx* ctx, const void* draft_logits, const void* target_logits,
                           const int32_t* d2t, const gto_tree* tree, float weight,
                           void* grad_root, const gto_token_stats* out, void* stream);
 
+/* The total loss of Sec. 3.2, L = L_token + omega * L_GTO, as ONE gradient buffer: the same
+ * computation as gto_token_loss, with the root-row gradient weight * (p_M - p_T) of position b
+ * going into slice grad[b,0,:] of the buffer gto_group_surrogate_grad filled ([B,D,V_draft]).
+ * Step 0 of an accepted path is always taken from the root row, so where that slice already
+ * holds a surrogate gradient (path_len[b] > 0 and coeff[b] != 0) the token gradient is added
+ * to it, and elsewhere the slice is overwritten.  Afterwards grad[b,0,:] is the derivative of
+ * weight * H_b + grad_scale * (sum of the group losses) with respect to the root row of
+ * position b, for every b (also where path_row[b,0] is -1).  Call it after
+ * gto_group_surrogate_grad on the same stream, with that call's reward and stats. */
+gto_status gto_token_loss_accumulate(gto_ctx* ctx, const void* draft_logits,
+                                     const void* target_logits, const int32_t* d2t,
+                                     const gto_tree* tree, const gto_reward* reward,
+                                     const gto_grad_stats* stats, float weight, void* grad,
+                                     const gto_token_stats* out, void* stream);
+
 /* SampleGroups of Algorithm 1 under Eq. 6-7: K non-overlapping groups of m adjacent positions
  * of a sequence of length s; start indices are 1-based, 1 <= t_k <= s - m + 1 and
  * t_{k+1} >= t_k + m.  Host-only (no device work): `u` is a HOST array of K uniforms in
- * [0, 1) supplied by the caller, `starts` a HOST array that receives t_1 < ... < t_K.  Every
- * admissible placement is equally likely for independent uniforms.  Returns
+ * [0, 1) supplied by the caller, `starts` a HOST array that receives t_1 < ... < t_K.  The
+ * paper fixes no law for the draw; this one turns the K uniforms into K independent offsets
+ * in [0, s - K m], sorts them and shifts the k-th (0-based) by k m.  Every admissible
+ * placement can occur, but not equally often: its weight is the number of orderings of its
+ * offsets, so placements with groups packed back to back (equal offsets) are rarer.  Returns
  * GTO_ERR_INVALID_ARG when K*m > s or an argument is out of range. */
 gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts);
 

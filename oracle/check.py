@@ -2,10 +2,12 @@
 (test infrastructure only).  Receives plain numpy arrays; imports nothing of the
 product path.
 
-Tolerances: integer structure bit-exact; a structural mismatch is excused only when
-the oracle's own ranking of that tree has a decision whose competing scores lie within
-1e-6 (counted and reported); rewards and advantages 1e-4 relative; gradients 2e-3
-absolute.
+Tolerances: integer structure bit-exact; a structural mismatch is excused only when the
+ranking decision that was resolved differently (a layer's frontier ranking, or the top-g
+cut) has competing oracle scores within 1e-6 (counted and reported); rewards, target
+probabilities and path products 1e-4 relative; advantages 1e-4 of max(1, |A|) (they amplify
+a reward error by 1 / std(R), so groups with std(R) < 1e-4 are reported as ill-conditioned
+and skipped); gradients 2e-3 absolute.
 """
 from __future__ import annotations
 
@@ -20,9 +22,47 @@ LSE_ATOL = 2e-6
 CLIP_EDGE_TOL = 1e-6
 
 
+SCORE_ATOL = 0.5 * TIE_TOL   # scores this close to the oracle's keep every decision whose gap is >= TIE_TOL
+
+
 def _close(a, b, rtol=REL_TOL, atol=0.0):
+    """|a - b| <= atol + rtol |b|, element by element (a true relative bound)."""
     a, b = np.asarray(a, dtype=np.float64), np.asarray(b, dtype=np.float64)
-    return np.all(np.abs(a - b) <= atol + rtol * np.maximum(1.0, np.abs(b)))
+    return np.all(np.abs(a - b) <= atol + rtol * np.abs(b))
+
+
+def differing_decisions(tr, got):
+    """Which ranking decisions of the oracle's tree `tr` the other side resolved differently,
+    with the oracle's score gap at each.  got: dict of the other side's node lists (pool, slot,
+    token, depth).  Looks at the shallowest depth whose selected nodes differ (deeper
+    differences follow from it): a node that is selected on one side only is the top-g cut;
+    a node selected on both sides with another frontier slot is that layer's ranking, and
+    the gap reported is the largest one between the ranks the disagreement spans.
+    Returns a list of (decision name, gap); empty if no ranking decision explains the
+    difference (then it is a plain error)."""
+    k = tr.k
+    out = []
+    for d in range(1, tr.D + 1):
+        mine = {int(p): (int(s), int(t)) for p, s, t, dd in zip(tr.pool, tr.slot, tr.token, tr.depth) if dd == d}
+        theirs = {int(p): (int(s), int(t)) for p, s, t, dd in
+                  zip(got["pool"], got["slot"], got["token"], got["depth"]) if dd == d}
+        if mine == theirs:
+            continue
+        if set(mine) != set(theirs):
+            out.append(("top-g cut", float(tr.cut_gaps[-1])))
+        both = [p for p in mine if p in theirs]
+        if any(mine[p][1] != theirs[p][1] for p in both):
+            return []                          # same candidate, other token: not a ranking matter
+        moved = [p for p in both if mine[p][0] != theirs[p][0]]
+        if moved:
+            if d not in tr.layer_gaps:
+                return []
+            rank = lambda s_: k if s_ < 0 else s_
+            ranks = [rank(mine[p][0]) for p in moved] + [rank(theirs[p][0]) for p in moved]
+            gaps = tr.layer_gaps[d][min(ranks):max(ranks)]
+            out.append((f"frontier ranking of depth {d}", float(max(gaps, default=np.inf))))
+        break
+    return out
 
 
 def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
@@ -41,7 +81,7 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
     assert n % m == 0
     agg = getattr(cfg, "agg", orc.AGG_LSE)
     rep = dict(positions=n, trees=G * n, near_tie_trees=0, clip_edge=0, ill_conditioned_groups=0,
-               max_lse_err=0.0, max_reward_rel=0.0, max_adv_err=0.0, max_grad_err=0.0,
+               max_lse_err=0.0, max_score_err=0.0, max_reward_rel=0.0, max_adv_err=0.0, max_grad_err=0.0,
                mean_path_len=0.0, mean_needed_rows=0.0)
     fwd = []
     excused = np.zeros(n, dtype=bool)
@@ -56,9 +96,10 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
                        [("node_token", "token"), ("node_parent", "parent"), ("node_depth", "depth"),
                         ("node_ctx_row", "ctx_row"), ("node_slot", "slot"), ("node_pool", "pool")])
             if not same:
-                gap = min(tr.cut_gaps)
-                assert gap < TIE_TOL, (f"tree structure mismatch at position {positions[i]} tree {t} "
-                                       f"with smallest decision gap {gap}")
+                why = differing_decisions(tr, dict(pool=gpu["node_pool"][t, i], slot=gpu["node_slot"][t, i],
+                                                   token=gpu["node_token"][t, i], depth=gpu["node_depth"][t, i]))
+                assert why and all(gap < TIE_TOL for _, gap in why), (
+                    f"tree structure mismatch at position {positions[i]} tree {t}: {why or 'no ranking decision differs'}")
                 rep["near_tie_trees"] += 1
                 excused[i] = True
                 continue
@@ -72,7 +113,9 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
             rep["max_lse_err"] = max(rep["max_lse_err"], float(err))
             assert err <= LSE_ATOL, f"draft lse error {err} at {positions[i]}"
             assert _close(gpu["node_logp"][t, i], tr.logp, rtol=0, atol=1e-5)
-            assert _close(gpu["node_score"][t, i], tr.score, rtol=0, atol=1e-5)
+            err = np.max(np.abs(gpu["node_score"][t, i] - tr.score))
+            rep["max_score_err"] = max(rep["max_score_err"], float(err))
+            assert err <= 1e-5, f"score error {err} at {positions[i]}"
             rw = f["rewards"][t]
             used = ~np.isnan(rw["row_lse_t"])
             assert np.array_equal(np.isnan(gpu["row_lse_t"][t, i]), ~used)
@@ -83,13 +126,14 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
             want_am = [orc.argmax_low(t_i[t, r]) for r in np.flatnonzero(used)]
             assert np.array_equal(gpu["row_argmax_t"][t, i][used], want_am)
             rep["mean_needed_rows"] += used.sum() / (G * n)
-            assert _close(gpu["node_ptarget"][t, i], rw["p"], rtol=REL_TOL, atol=1e-12)
-            assert _close(gpu["node_pathprod"][t, i], rw["Pp"], rtol=REL_TOL, atol=1e-12)
-            assert _close(gpu["node_L"][t, i], rw["Lc"])
-            rel = abs(gpu["reward"][t, i] - rw["r"]) / max(1.0, abs(rw["r"]))
+            # stored as fp32: values below the smallest normal number may flush
+            assert _close(gpu["node_ptarget"][t, i], rw["p"], atol=1e-37)
+            assert _close(gpu["node_pathprod"][t, i], rw["Pp"], atol=1e-37)
+            assert _close(gpu["node_L"][t, i], rw["Lc"], atol=1e-37)
+            rel = abs(gpu["reward"][t, i] - rw["r"]) / max(1e-7, abs(rw["r"]))
             rep["max_reward_rel"] = max(rep["max_reward_rel"], float(rel))
             assert rel <= REL_TOL, f"reward {gpu['reward'][t, i]} vs {rw['r']}"
-            assert _close(gpu["etree"][t, i], rw["etree"])
+            assert _close(gpu["etree"][t, i], rw["etree"], atol=1e-37)
             assert gpu["n_leaves"][t, i] == len(rw["leaves"])
         if excused[i]:
             continue
@@ -127,19 +171,22 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
             path_tok[j, :l] = fwd[i]["path"]["tokens"]
         old = old_logp_fn(path_logp, path_row, path_tok, path_len, [positions[i] for i in idx])
         sur = orc.clipped_surrogate(path_logp, old, path_len, A, m, cfg.clip_eps, cfg.grad_scale)
-        assert _close(gpu["R"][idx], R, rtol=REL_TOL)
+        # a difference of two rewards: relative to the rewards, not to the difference
+        assert np.all(np.abs(gpu["R"][idx] - R) <= REL_TOL * np.maximum(np.abs(r_cur), np.abs(r_ref)))
         adv_err = np.max(np.abs(gpu["adv"][idx] - A) / np.maximum(1.0, np.abs(A)))
         rep["max_adv_err"] = max(rep["max_adv_err"], float(adv_err))
         assert adv_err <= REL_TOL, f"advantage error {adv_err}"
-        assert _close(gpu["ratio"][idx], sur["ratio"])
+        assert _close(gpu["ratio"][idx], sur["ratio"])          # s > 0: a relative bound
         edge = np.minimum(np.abs(sur["ratio"] - (1 + cfg.clip_eps)),
                           np.abs(sur["ratio"] - (1 - cfg.clip_eps))) < CLIP_EDGE_TOL
         rep["clip_edge"] += int(edge.sum())
         if edge.any():
             continue
         assert np.array_equal(gpu["active"][idx].astype(bool), sur["active"])
-        assert _close(gpu["coeff"][idx], sur["coeff"], rtol=REL_TOL, atol=1e-9)
-        assert _close(gpu["loss"][g0 // m], sur["loss"][0], rtol=REL_TOL, atol=1e-9)
+        # coefficients and the group loss are sums over advantages: 1e-4 of the advantages' scale
+        scale = REL_TOL * float(np.max(np.abs(A) * sur["ratio"])) / m
+        assert _close(gpu["coeff"][idx], sur["coeff"], rtol=REL_TOL, atol=abs(cfg.grad_scale) * scale)
+        assert _close(gpu["loss"][g0 // m], sur["loss"][0], rtol=REL_TOL, atol=m * scale)
         for j, i in enumerate(idx):
             l = path_len[j]
             d_i = np.asarray(draft[0, i], dtype=np.float64)
@@ -149,5 +196,6 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
                                            draft.shape[-1])
             err = float(np.max(np.abs(gpu["grad"][i] - want)))
             rep["max_grad_err"] = max(rep["max_grad_err"], err)
-            assert err <= GRAD_ATOL, f"gradient error {err} at position {positions[i]}"
+            # 2e-3 absolute is stated for grad_scale = 1; entries scale with it
+            assert err <= GRAD_ATOL * abs(cfg.grad_scale), f"gradient error {err} at position {positions[i]}"
     return rep

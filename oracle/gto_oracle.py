@@ -91,6 +91,7 @@ class DraftTree:
     mask: np.ndarray       # [g,g] bool, mask[n,a] = a is n or an ancestor of n
     row_lse: np.ndarray    # [R] draft log-sum-exp of every context row
     cut_gaps: list = field(default_factory=list)  # smallest score gap behind each layer ranking and the top-g cut
+    layer_gaps: dict = field(default_factory=dict)  # depth d -> gaps between ranks (r, r+1), r < k, of layer d's ranking
 
 
 def context_row(d, j, k):
@@ -105,12 +106,19 @@ def draft_slot_of_row(r, k):
 
 
 def _decision_gap(pool, a, b):
-    """Score gap between two candidates that a ranking decision separates.  Two
-    children of one parent with the same logit tie exactly on every implementation
-    (the index decides), so that case is not a fragile decision: report inf."""
+    """Score gap between two candidates that a ranking decision separates (a ranked first).
+    Two cases are decided by the index on every implementation and are not fragile, so they
+    report inf: two children of one parent with the same logit (their scores are the same
+    sum), and a candidate against its own descendant (a log-probability is never positive,
+    so the descendant cannot score higher, and on a tie the ancestor has the lower index)."""
     gap = pool[a]["score"] - pool[b]["score"]
     if gap == 0.0 and pool[a]["parent_pool"] == pool[b]["parent_pool"]:
         return np.inf
+    up = pool[b]["parent_pool"]
+    while up >= 0:
+        if up == a:
+            return np.inf
+        up = pool[up]["parent_pool"]
     return gap
 
 
@@ -135,6 +143,7 @@ def build_tree(draft, D, k, g):
     pool = []          # pool[p] = dict(score, logp, depth, ctx_row, token, parent_pool)
     slot_of = {}       # pool index -> frontier slot
     cut_gaps = []
+    layer_gaps = {}
 
     lse, ids, lp = lse_and_topk(draft[0, 0], k)
     row_lse[0] = lse
@@ -159,8 +168,9 @@ def build_tree(draft, D, k, g):
             layer.sort(key=lambda p: (-pool[p]["score"], p))
             frontier = layer[:k]
             # slots are ranks, so every adjacent pair down to the cut is a decision
-            cut_gaps.append(min([_decision_gap(pool, layer[r], layer[r + 1])
-                                 for r in range(min(k, len(layer) - 1))], default=np.inf))
+            layer_gaps[d] = [_decision_gap(pool, layer[r], layer[r + 1])
+                             for r in range(min(k, len(layer) - 1))]
+            cut_gaps.append(min(layer_gaps[d], default=np.inf))
             for j, p in enumerate(frontier):
                 slot_of[p] = j
     assert len(pool) == P
@@ -190,7 +200,8 @@ def build_tree(draft, D, k, g):
         mask[n, n] = True
     return DraftTree(D=D, k=k, g=g, token=token, parent=parent, depth=depth, ctx_row=ctx,
                      slot=slot, pool=np.array(selected, dtype=np.int64), logp=logp,
-                     score=score, mask=mask, row_lse=row_lse, cut_gaps=cut_gaps)
+                     score=score, mask=mask, row_lse=row_lse, cut_gaps=cut_gaps,
+                     layer_gaps=layer_gaps)
 
 
 # ------------------------------------------------------------------------ O5-O6
@@ -457,9 +468,11 @@ def sample_groups(s, m, K, u):
     """SampleGroups of Algorithm 1 under the constraints of Eq. 6-7: K non-overlapping
     groups of m adjacent positions of a sequence of length s, start indices 1-based with
     1 <= t_k <= s - m + 1 and t_{k+1} >= t_k + m.  The paper does not say how the starts
-    are drawn; here every admissible placement is equally likely: the K uniforms u in
-    [0, 1) are turned into integers in [0, s - K m], sorted, and the k-th (0-based) is
-    shifted by k m.  Returns the start indices t_1 < ... < t_K.
+    are drawn; here the K uniforms u in [0, 1) are turned into K independent integer offsets
+    in [0, s - K m], sorted, and the k-th (0-based) is shifted by k m.  Every admissible
+    placement can occur; its probability is proportional to the number of orderings of its
+    offsets (placements with equal offsets, i.e. groups back to back, are rarer).
+    Returns the start indices t_1 < ... < t_K.
     """
     assert K >= 0 and m >= 1 and K * m <= s
     free = s - K * m

@@ -75,6 +75,10 @@ _lib.gto_group_surrogate_grad.argtypes = [_vp, _vp, ctypes.POINTER(gto_tree), ct
 _lib.gto_token_loss.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(gto_tree), ctypes.c_float, _vp,
                                 ctypes.POINTER(gto_token_stats), _vp]
 _lib.gto_token_loss.restype = ctypes.c_int
+_lib.gto_token_loss_accumulate.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(gto_tree),
+                                           ctypes.POINTER(gto_reward), ctypes.POINTER(gto_grad_stats),
+                                           ctypes.c_float, _vp, ctypes.POINTER(gto_token_stats), _vp]
+_lib.gto_token_loss_accumulate.restype = ctypes.c_int
 _lib.gto_sample_groups.argtypes = [ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
                                    ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int32)]
 _lib.gto_sample_groups.restype = ctypes.c_int
@@ -238,6 +242,25 @@ def gto_token_loss(ctx: int, draft: torch.Tensor, target: torch.Tensor, d2t, tre
                                _stream_ptr(stream)), "gto_token_loss")
 
 
+def gto_token_loss_accumulate(ctx: int, draft: torch.Tensor, target: torch.Tensor, d2t, tree: dict,
+                              reward: dict, stats: dict, weight: float, grad: torch.Tensor,
+                              token_stats: dict, stream=None):
+    """gto_token_loss into slice [b, 0, :] of the surrogate's gradient buffer [B, D, V_draft]."""
+    assert draft.is_cuda and draft.is_contiguous() and target.is_cuda and target.is_contiguous()
+    assert grad.is_cuda and grad.is_contiguous() and grad.dtype == draft.dtype and grad.dim() == 3
+    if d2t is not None:
+        assert d2t.is_cuda and d2t.dtype == torch.int32 and d2t.is_contiguous()
+    t = _fill(gto_tree, _TREE_FIELDS, tree)
+    r = _fill(gto_reward, _REWARD_FIELDS, reward)
+    g = _fill(gto_grad_stats, _STATS_FIELDS, stats)
+    s = _fill(gto_token_stats, _TOKEN_FIELDS, token_stats)
+    _check(_lib.gto_token_loss_accumulate(ctx, draft.data_ptr(), target.data_ptr(),
+                                          None if d2t is None else d2t.data_ptr(), ctypes.byref(t),
+                                          ctypes.byref(r), ctypes.byref(g), ctypes.c_float(weight),
+                                          grad.data_ptr(), ctypes.byref(s), _stream_ptr(stream)),
+           "gto_token_loss_accumulate")
+
+
 def gto_sample_groups(s: int, m: int, K: int, u) -> list:
     """Start indices (1-based) of K non-overlapping groups of m adjacent positions (host only)."""
     uu = (ctypes.c_double * max(K, 1))(*[float(x) for x in list(u)[:K]])
@@ -275,4 +298,5 @@ def gto_kernel_times(ctx: int, stream=None) -> dict:
 
 EXPORTS = ["gto_create", "gto_destroy", "gto_build_tree", "gto_tree_reward",
            "gto_group_surrogate_grad", "gto_device_status", "gto_launch_count", "gto_status_string",
-           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss", "gto_sample_groups", "gto_tree_reward_host"]
+           "gto_kernel_timing", "gto_kernel_times", "gto_build_tree_noalloc", "gto_token_loss", "gto_sample_groups", "gto_tree_reward_host",
+           "gto_token_loss_accumulate"]

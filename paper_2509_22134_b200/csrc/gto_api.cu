@@ -21,6 +21,10 @@ struct gto_ctx {
   int32_t* list;      // [G*B*R] needed target rows
   int32_t* list_count;
   int32_t* status;
+  uint32_t* map_bits;   // token loss: bitmap of the id map's image, and
+  uint32_t* map_prefix; //   the number of mapped ids below each of its words
+  int32_t* map_state;   //   [0] = 1 if the map is not increasing
+  int sms;
   int32_t* h_list;    // page-locked host copy of the work list: [0] = count, then the rows
   int64_t last_host_rows;
   int64_t launches;
@@ -165,6 +169,7 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
       delete ctx;
       return GTO_ERR_CUDA;
     }
+    ctx->sms = sms;
     ctx->row_grid_cap = sms * 12 * GTO_ROW_GRID_WAVES;
     ctx->row_split_rows = sms * GTO_ROW_SPLIT_ROWS_PER_SM;
   }
@@ -175,8 +180,12 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   const size_t o_id = off;  off += align_up(rows * c->k * sizeof(int32_t));
   const size_t o_z = off;   off += align_up(rows * c->k * sizeof(float));
   const size_t o_list = off; off += align_up(rows * sizeof(int32_t));
+  const size_t map_words = static_cast<size_t>(c->V_target + 31) / 32 + 1;
+  const size_t o_bits = off; off += align_up(map_words * sizeof(uint32_t));
+  const size_t o_pre = off; off += align_up(map_words * sizeof(uint32_t));
   const size_t o_cnt = off; off += 256;
   const size_t o_st = off;  off += 256;
+  const size_t o_ms = off;  off += 256;
   if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
     cudaGetLastError();
     delete ctx;
@@ -187,7 +196,10 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->list = reinterpret_cast<int32_t*>(ctx->ws + o_list);
   ctx->list_count = reinterpret_cast<int32_t*>(ctx->ws + o_cnt);
   ctx->status = reinterpret_cast<int32_t*>(ctx->ws + o_st);
-  if (cudaMemset(ctx->ws + o_cnt, 0, 512) != cudaSuccess ||
+  ctx->map_bits = reinterpret_cast<uint32_t*>(ctx->ws + o_bits);
+  ctx->map_prefix = reinterpret_cast<uint32_t*>(ctx->ws + o_pre);
+  ctx->map_state = reinterpret_cast<int32_t*>(ctx->ws + o_ms);
+  if (cudaMemset(ctx->ws + o_cnt, 0, 768) != cudaSuccess ||
       cudaMallocHost(&ctx->h_list, (rows + 1) * sizeof(int32_t)) != cudaSuccess) {
     cudaGetLastError();
     cudaFree(ctx->ws);
@@ -396,12 +408,15 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
   return GTO_OK;
 }
 
-gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, const int32_t* d2t,
-                          const gto_tree* tree, float weight, void* grad_root,
-                          const gto_token_stats* out, void* stream) {
-  CallRange range("gto_token_loss");
-  if (!ctx || !draft || !target || !tree || !grad_root || !out || !aligned16(draft) ||
-      !aligned16(target) || !aligned16(grad_root) || !all_set(tree) || !all_set(out))
+namespace {
+
+// Shared body of gto_token_loss and gto_token_loss_accumulate.
+gto_status token_loss_impl(gto_ctx* ctx, const void* draft, const void* target, const int32_t* d2t,
+                           const gto_tree* tree, float weight, void* grad_out, int64_t out_stride,
+                           const int32_t* acc_path_len, const double* acc_coeff,
+                           const gto_token_stats* out, void* stream) {
+  if (!ctx || !draft || !target || !tree || !grad_out || !out || !aligned16(draft) ||
+      !aligned16(target) || !aligned16(grad_out) || !all_set(tree) || !all_set(out))
     return GTO_ERR_INVALID_ARG;
   const gto_config& c = ctx->cfg;
   if (!d2t && c.V_draft != c.V_target) return GTO_ERR_INVALID_ARG;
@@ -416,13 +431,42 @@ gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, c
   a.target = target;
   a.d2t = d2t;
   a.row_lse = tree->row_lse;
-  a.grad_root = grad_root;
+  a.grad_out = grad_out;
+  a.out_stride = out_stride;
+  a.acc_path_len = acc_path_len;
+  a.acc_coeff = acc_coeff;
   a.loss = out->loss;
   a.lse_t = out->lse_t;
   a.status = ctx->status;
+  a.map_bits = ctx->map_bits;
+  a.map_prefix = ctx->map_prefix;
+  a.map_state = ctx->map_state;
   LaunchSpan span(ctx, GTO_K_TOKEN_LOSS, s);
-  if (gto::launch_token_loss(a, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
+  if (gto::launch_token_loss(a, ctx->sms, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;
+}
+
+}  // namespace
+
+gto_status gto_token_loss(gto_ctx* ctx, const void* draft, const void* target, const int32_t* d2t,
+                          const gto_tree* tree, float weight, void* grad_root,
+                          const gto_token_stats* out, void* stream) {
+  CallRange range("gto_token_loss");
+  if (!ctx) return GTO_ERR_INVALID_ARG;
+  return token_loss_impl(ctx, draft, target, d2t, tree, weight, grad_root, ctx->cfg.V_draft, nullptr,
+                         nullptr, out, stream);
+}
+
+gto_status gto_token_loss_accumulate(gto_ctx* ctx, const void* draft, const void* target,
+                                     const int32_t* d2t, const gto_tree* tree,
+                                     const gto_reward* reward, const gto_grad_stats* stats,
+                                     float weight, void* grad, const gto_token_stats* out,
+                                     void* stream) {
+  CallRange range("gto_token_loss_accumulate");
+  if (!ctx || !reward || !stats || !all_set(reward) || !all_set(stats)) return GTO_ERR_INVALID_ARG;
+  return token_loss_impl(ctx, draft, target, d2t, tree, weight, grad,
+                         static_cast<int64_t>(ctx->cfg.D) * ctx->cfg.V_draft, reward->path_len,
+                         stats->coeff, out, stream);
 }
 
 gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts) {

@@ -45,6 +45,12 @@ struct Bf16 {
   static constexpr int kPerVec = 8;
   static constexpr int kBytes = 2;
   static constexpr uint32_t kNegInfWord = 0xff80ff80u;
+  using Storage = uint16_t;
+  // stored bits of element e of a vector
+  __device__ static __forceinline__ Storage element(const uint4& v, int e) {
+    const uint32_t w = e < 4 ? (e < 2 ? v.x : v.y) : (e < 6 ? v.z : v.w);
+    return static_cast<Storage>(e & 1 ? w >> 16 : w & 0xffffu);
+  }
   __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
     f[0] = __uint_as_float(v.x << 16);
     f[1] = __uint_as_float(v.x & 0xffff0000u);
@@ -90,6 +96,11 @@ struct F16 {
   static constexpr int kPerVec = 8;
   static constexpr int kBytes = 2;
   static constexpr uint32_t kNegInfWord = 0xfc00fc00u;
+  using Storage = uint16_t;
+  __device__ static __forceinline__ Storage element(const uint4& v, int e) {
+    const uint32_t w = e < 4 ? (e < 2 ? v.x : v.y) : (e < 6 ? v.z : v.w);
+    return static_cast<Storage>(e & 1 ? w >> 16 : w & 0xffffu);
+  }
   __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -132,6 +143,10 @@ struct F32 {
   static constexpr int kPerVec = 4;
   static constexpr int kBytes = 4;
   static constexpr uint32_t kNegInfWord = 0xff800000u;
+  using Storage = uint32_t;
+  __device__ static __forceinline__ Storage element(const uint4& v, int e) {
+    return e < 2 ? (e == 0 ? v.x : v.y) : (e == 2 ? v.z : v.w);
+  }
   __device__ static __forceinline__ void unpack(const uint4& v, float (&f)[4]) {
     f[0] = __uint_as_float(v.x);
     f[1] = __uint_as_float(v.y);

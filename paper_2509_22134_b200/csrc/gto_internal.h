@@ -87,12 +87,19 @@ struct TokenLossArgs {
   const void* target;      // [G,B,R,V_target]; row [0,b,0,:] is read
   const int32_t* d2t;      // [V_draft] or null (identity)
   const double* row_lse;   // [G*B*R] draft log-sum-exp (entry of row 0 of tree (0,b))
-  void* grad_root;         // [B, V_draft] in the logit dtype
+  void* grad_out;          // gradient rows in the logit dtype: row b starts at b * out_stride
+  int64_t out_stride;      // elements between the rows of consecutive positions
+  const int32_t* acc_path_len;  // accumulate mode: [B] accepted lengths, else null
+  const double* acc_coeff;      // accumulate mode: [B] surrogate coefficients
   double* loss;            // [B]
   double* lse_t;           // [B]
   int32_t* status;
+  uint32_t* map_bits;      // workspace: bitmap of the id map's image, ceil(V_target/32)+1 words
+  uint32_t* map_prefix;    // workspace: mapped ids below each bitmap word
+  int32_t* map_state;      // workspace: [0] = 1 if the map is not increasing
 };
-cudaError_t launch_token_loss(const TokenLossArgs& a, cudaStream_t stream, int64_t* launches);
+cudaError_t launch_token_loss(const TokenLossArgs& a, int sms, cudaStream_t stream,
+                              int64_t* launches);
 
 cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches);

@@ -12,8 +12,11 @@
 // number of entries ahead of it (a binary search again); only the first g of a layer can
 // reach the global top-g.  Ties go to the lower index everywhere: child index within a
 // parent, parent slot within a layer, layer (= depth) across layers, i.e. the pool index.
-// Scores are fp64 sums of (z - lse), so a ranking differs from an exact evaluation only
-// where two scores agree to ~1e-7.
+// Scores are fp64 sums of min(z - lse, 0), so a ranking differs from an exact evaluation only
+// where two scores agree to ~1e-7.  The clamp matters: a log-probability is never positive,
+// but the fp32-accumulated log-sum-exp of a row with one dominant logit can come out a few
+// 1e-7 below that logit; without the clamp such a child would outscore its own parent and
+// could be kept by the prune without it.
 #include "gto_common.cuh"
 #include "gto_internal.h"
 
@@ -24,6 +27,11 @@ constexpr int kTreeThreads = 128;
 static_assert(kMaxLayer <= kTreeThreads, "one thread per layer candidate");
 static_assert(kMaxNodes <= kTreeThreads, "one thread per selected node");
 constexpr int kMaskWords = kMaxLayer / 32;
+
+// Draft log-probability of a listed token: z - lse, never above 0.
+__device__ __forceinline__ double edge_logp(float z, double lse) {
+  return fmin(static_cast<double>(z) - lse, 0.0);
+}
 
 __device__ __forceinline__ uint64_t score_key(double s) {
   uint64_t u = static_cast<uint64_t>(__double_as_longlong(s + 0.0));
@@ -111,7 +119,7 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
   __syncthreads();
   // ---- depth 1: the root's k best tokens, already in rank order = pool order
   if (tid < k) {
-    const double sc = static_cast<double>(top_z[tid]) - lse[0];
+    const double sc = edge_logp(top_z[tid], lse[0]);
     skey[tid] = score_key(sc);
     sq[tid] = static_cast<uint8_t>(tid);
     if (D > 1) {
@@ -130,7 +138,7 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
     uint64_t key = 0;
     if (tid < kk) {
       const int row = 1 + (d - 2) * k + j;
-      sc = sm.fcum[cur][j] + (static_cast<double>(top_z[row * k + c]) - lse[row]);
+      sc = sm.fcum[cur][j] + edge_logp(top_z[row * k + c], lse[row]);
       key = score_key(sc);
       sm.ukey[tid] = key;
     }
@@ -224,8 +232,7 @@ __global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs 
     a.out.node_ctx_row[obase + n] = ctx;
     a.out.node_slot[obase + n] = (depth < D && r < k) ? r : -1;  // frontier slot = layer rank
     a.out.node_pool[obase + n] = off + q;
-    a.out.node_logp[obase + n] =
-        static_cast<float>(static_cast<double>(top_z[ctx * k + c]) - lse[ctx]);
+    a.out.node_logp[obase + n] = static_cast<float>(edge_logp(top_z[ctx * k + c], lse[ctx]));
     a.out.node_score[obase + n] = key_score(skey[off + r]);
   }
   __syncthreads();

@@ -76,6 +76,13 @@ class GtoPass:
         gto.gto_token_loss(self.ctx, draft, target, d2t, self.tree, weight, self.grad_root,
                            self.token_stats, stream)
 
+    def token_loss_accumulate(self, draft, target, d2t, weight: float = 1.0, stream=None):
+        """Token-level loss added into slice [b, 0, :] of the surrogate gradient buffer."""
+        if not hasattr(self, "token_stats"):
+            self.token_stats = gto.alloc_token_stats(self.cfg, self.device)
+        gto.gto_token_loss_accumulate(self.ctx, draft, target, d2t, self.tree, self.reward, self.stats,
+                                      weight, self.grad, self.token_stats, stream)
+
     def status(self) -> int:
         return gto.gto_device_status(self.ctx)
 

@@ -15,3 +15,12 @@ def pytest_configure(config):
 @pytest.fixture(scope="session")
 def repo_root():
     return ROOT
+
+
+@pytest.fixture(scope="session")
+def oracle_workers():
+    """Worker processes that run the oracle on every host core (full-size parity checks)."""
+    from oracle.parallel import OracleWorkers
+    pool = OracleWorkers(min(os.cpu_count() or 1, 16), extra_sys_path=[os.path.join(ROOT, "tests")])
+    yield pool
+    pool.close()

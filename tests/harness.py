@@ -8,7 +8,8 @@ from __future__ import annotations
 import numpy as np
 import torch
 
-from oracle import check as ocheck
+import oracle_tasks
+from oracle import parallel as opar
 from paper_2509_22134_b200 import synth
 from paper_2509_22134_b200.runner import GtoPass
 
@@ -46,28 +47,20 @@ def run_pass(w: synth.Workload, device="cuda:0", data=None, **kw):
     return p, data
 
 
-def check_against_oracle(w: synth.Workload, p: GtoPass, data, groups, cfg_extra=None):
-    """Oracle comparison on the listed groups (each m consecutive positions)."""
-    pos = [gidx * w.m + i for gidx in groups for i in range(w.m)]
-    idx = torch.as_tensor(pos, device=p.device, dtype=torch.long)
-    draft = data["draft"].index_select(1, idx).float().cpu().numpy()
-    target = data["target"].index_select(1, idx).float().cpu().numpy()
+def check_against_oracle(w: synth.Workload, p: GtoPass, data, groups, cfg_extra=None, workers=None):
+    """Oracle comparison on the listed groups (each m consecutive positions).  With `workers`
+    (an oracle.parallel.OracleWorkers) every group is checked on its own host core."""
     d2t = None if data["d2t"] is None else data["d2t"].cpu().numpy().astype(np.int64)
-    gpu = gather_outputs(p, pos)
 
-    class Cfg:
-        pass
-    cfg = Cfg()
-    for name in ("B", "G", "D", "k", "g", "m", "eta", "clip_eps", "std_delta", "grad_scale"):
-        setattr(cfg, name, getattr(w, name))
-    for key, val in (cfg_extra or {}).items():
-        setattr(cfg, key, val)
+    def payload(gs):
+        pos = [gidx * w.m + i for gidx in gs for i in range(w.m)]
+        idx = torch.as_tensor(pos, device=p.device, dtype=torch.long)
+        draft, dtag = opar.encode_logits(data["draft"].index_select(1, idx))
+        target, ttag = opar.encode_logits(data["target"].index_select(1, idx))
+        return dict(w=w, cfg_extra=cfg_extra, draft=draft, draft_tag=dtag, target=target,
+                    target_tag=ttag, d2t=d2t, gpu=gather_outputs(p, pos), positions=pos)
 
-    def old_fn(path_logp, path_row, path_token, path_len, positions):
-        out = np.zeros_like(path_logp)
-        for j, b in enumerate(positions):
-            out[j] = synth.old_logp_from_path(w, path_logp[j:j + 1], path_row[j:j + 1],
-                                              path_token[j:j + 1], path_len[j:j + 1], b0=b)[0]
-        return out
-
-    return ocheck.check_positions(cfg, draft, target, d2t, gpu, old_fn, pos)
+    if workers is None or len(groups) == 1:
+        return oracle_tasks.check_groups(**payload(list(groups)))
+    reps, _ = workers.run("oracle_tasks", "check_groups", [payload([gidx]) for gidx in groups])
+    return oracle_tasks.merge_reports(reps)

@@ -1,0 +1,99 @@
+"""The comparison harness itself (oracle/check.py): a structural mismatch is excused only by
+the ranking decision that was actually resolved differently, never by an unrelated near tie."""
+import numpy as np
+import pytest
+
+from oracle import check as ocheck
+from oracle import gto_oracle as orc
+
+D, K, G_NODES, V = 4, 3, 12, 12
+
+
+def lists(tree):
+    return dict(pool=tree.pool, slot=tree.slot, token=tree.token, depth=tree.depth)
+
+
+def candidate_site(tree_draft, tree, node):
+    """(d, j, token) of the draft logit that feeds the edge into `node`."""
+    d, j = orc.draft_slot_of_row(int(tree.ctx_row[node]), K)
+    return d, j, int(tree.token[node])
+
+
+def find_case(kind):
+    """A random tree plus a copy of its logits with ONE logit raised just enough to flip one
+    decision: two adjacent frontier ranks of a layer, or the top-g cut."""
+    for seed in range(200):
+        rng = np.random.default_rng(seed)
+        draft = rng.normal(size=(D, K, V)) * 2.0
+        tr = orc.build_tree(draft, D, K, G_NODES)
+        if kind == "layer":
+            d = 2 + seed % (D - 2)
+            nodes = [n for n in range(tr.g) if tr.depth[n] == d and tr.slot[n] >= 0]
+            by_slot = {int(tr.slot[n]): n for n in nodes}
+            pairs = [r for r in range(K - 1) if r in by_slot and r + 1 in by_slot]
+            if not pairs:
+                continue
+            r = pairs[0]
+            lower = by_slot[r + 1]
+            gap = tr.layer_gaps[d][r]
+            site = candidate_site(draft, tr, lower)
+            p_edge = np.exp(tr.logp[lower])
+        else:
+            gap = tr.cut_gaps[-1]
+            # the best unselected candidate: rebuild with one more node to learn where it sits
+            bigger = orc.build_tree(draft, D, K, G_NODES + 1)
+            extra = [n for n in range(bigger.g) if bigger.pool[n] not in set(tr.pool)]
+            if len(extra) != 1:
+                continue
+            site = candidate_site(draft, bigger, extra[0])
+            p_edge = np.exp(bigger.logp[extra[0]])
+            d, r = None, None
+        if not (1e-3 < gap < 0.3):
+            continue
+        bumped = draft.copy()
+        bumped[site] += gap * 1.2 / (1.0 - p_edge)     # raises the edge's log-probability by 1.2 gap
+        other = orc.build_tree(bumped, D, K, G_NODES)
+        if kind == "layer":
+            # keep the case only if the bump did exactly what was meant: same nodes down to
+            # depth d, with the slots of the two chosen nodes exchanged
+            upto = lambda t: {int(p): int(s) for p, s, dd in zip(t.pool, t.slot, t.depth) if dd <= d}
+            want = upto(tr)
+            a, b = int(tr.pool[by_slot[r]]), int(tr.pool[lower])
+            want[a], want[b] = want[b], want[a]
+            if upto(other) != want:
+                continue
+        else:
+            if len(set(other.pool) - set(tr.pool)) != 1 or not np.array_equal(
+                    other.slot[np.isin(other.pool, tr.pool)], tr.slot[np.isin(tr.pool, other.pool)]):
+                continue
+        why = ocheck.differing_decisions(tr, lists(other))
+        return tr, other, why, gap, d
+    raise AssertionError("no case found")
+
+
+def test_a_flipped_frontier_ranking_is_named_with_its_own_gap():
+    tr, other, why, gap, d = find_case("layer")
+    assert len(why) == 1 and why[0][0] == f"frontier ranking of depth {d}"
+    assert why[0][1] == pytest.approx(gap, rel=1e-12)
+    assert min(tr.cut_gaps) <= gap          # an unrelated, smaller gap may exist: it must not excuse
+
+
+def test_a_flipped_top_g_cut_is_named_with_its_own_gap():
+    tr, other, why, gap, _ = find_case("cut")
+    assert why == [("top-g cut", pytest.approx(gap, rel=1e-12))]
+
+
+def test_identical_trees_and_plain_errors():
+    rng = np.random.default_rng(7)
+    tr = orc.build_tree(rng.normal(size=(D, K, V)) * 2.0, D, K, G_NODES)
+    assert ocheck.differing_decisions(tr, lists(tr)) == []
+    wrong = lists(tr)
+    wrong["token"] = tr.token.copy()
+    wrong["token"][3] += 1                  # same candidate, another token: no ranking explains it
+    assert ocheck.differing_decisions(tr, wrong) == []
+
+
+def test_relative_bound_has_no_floor():
+    assert ocheck._close([1.00005e-3], [1e-3])
+    assert not ocheck._close([1.1e-3], [1e-3])          # 10 % off on a small probability
+    assert not ocheck._close([2e-9], [1e-9])

@@ -129,9 +129,10 @@ def test_ratio_is_one_when_old_equals_current_and_clip_edges():
     assert sur["active"].all()
 
 
-def test_sample_groups_respects_the_constraints_and_is_uniform_over_placements():
-    """Eq. 6-7: 1 <= t_k <= s - m + 1, t_{k+1} >= t_k + m.  Brute force on a tiny case: every
-    admissible placement is hit equally often when the uniforms sweep a fine grid."""
+def test_sample_groups_respects_the_constraints_and_reaches_every_placement():
+    """Eq. 6-7: 1 <= t_k <= s - m + 1, t_{k+1} >= t_k + m.  Brute force on a tiny case: when
+    the uniforms sweep a fine grid every admissible placement is produced, each as often as
+    its offsets have orderings (the law of K independent sorted offsets: valid, not uniform)."""
     import itertools
     s, m, K = 9, 2, 3
     placements = [t for t in itertools.combinations(range(1, s - m + 2), K)

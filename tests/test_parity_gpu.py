@@ -115,6 +115,31 @@ def test_variants_max_mean_unbiased_nodebias(harness):
     p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_SEQ_ALL_NODES)
     rep = harness.check_against_oracle(w, p, data, groups=[0, 1], cfg_extra=dict(all_nodes=True))
     assert int(p.reward["n_leaves"].min()) == w.g
+    from dataclasses import replace
+    w4 = replace(w, eta=4.0)          # the all-nodes reading at another temperature
+    p, data = harness.run_pass(w4, DEV, flags=gto.GTO_FLAG_SEQ_ALL_NODES)
+    harness.check_against_oracle(w4, p, data, groups=[0, 1], cfg_extra=dict(all_nodes=True))
+
+
+@pytest.mark.parametrize("grad_scale", [1.0, 0.5 / 16])
+@pytest.mark.parametrize("std_delta", [1e-6, 1e-2])
+@pytest.mark.parametrize("clip_eps", [0.05, 0.2, 0.5])
+@pytest.mark.parametrize("eta", [0.25, 1.0, 4.0])
+def test_hyper_parameters_away_from_their_defaults(harness, eta, clip_eps, std_delta, grad_scale):
+    """Smooth-max temperature (Eq. 5), delta of Eq. 10, epsilon of Eq. 12 and the factor on
+    the summed group losses all come from the configuration: every combination through the
+    oracle.  The narrow clip range leaves some ratios outside it, the wide one none."""
+    w = synth.Workload("hyper", B=32, V_draft=4104, V_target=4104, D=5, k=6, g=40, seed=606,
+                       eta=eta, clip_eps=clip_eps, std_delta=std_delta, grad_scale=grad_scale,
+                       old_sigma=0.12)
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=list(range(w.B // w.m)))
+    active = p.stats["active"].bool()
+    live = p.reward["path_len"] > 0
+    if clip_eps == 0.05:
+        assert bool((~active & live).any()) and bool((active & live).any())
+    assert float(p.stats["coeff"].abs().max()) <= abs(grad_scale) * 3.0
+    print(rep)
 
 
 @pytest.mark.parametrize("D,g", [(6, 50), (6, 70), (7, 50), (7, 70), (8, 50), (8, 60), (8, 70)])
@@ -185,6 +210,88 @@ def test_token_loss_matches_the_oracle(harness, kw):
         assert abs(loss[b] - H) <= 1e-4 * max(1.0, abs(H)), (b, loss[b], H)
         err = np.abs(grad[b] - weight * g)
         assert np.all(err <= 2e-3 * weight + 2.0 ** -8 * np.abs(weight * g)), (b, err.max())
+
+
+def _token_loss_reference(w, data, d2t):
+    from oracle import gto_oracle as orc
+    zd = data["draft"][0, :, 0, 0].float().cpu().numpy()
+    zt = data["target"][0, :, 0].float().cpu().numpy()
+    return [orc.token_loss(zd[b], zt[b], d2t) for b in range(w.B)]
+
+
+@pytest.mark.parametrize("kw", [
+    dict(B=8, V_draft=2048, V_target=8200, D=2, k=4, g=8, dtype="bf16", seed=26),      # cluster of 8
+    dict(B=640, V_draft=2048, V_target=8200, D=2, k=4, g=8, dtype="bf16", seed=27),    # one CTA per position
+    dict(B=8, V_draft=40000, V_target=40000, D=2, k=4, g=8, dtype="f32", seed=28),     # 160 KB rows, no map
+    dict(B=8, V_draft=1000, V_target=5000, D=2, k=4, g=8, dtype="f32", seed=29),       # fp32 with a map
+    dict(B=8, V_draft=8, V_target=64, D=2, k=2, g=4, dtype="bf16", seed=30),           # fewer vectors than CTAs
+])
+def test_token_loss_streaming_layouts(harness, kw):
+    """Eq. 13 through the streaming kernel at every cluster size, with empty and ragged ranges."""
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.Workload("tok", **kw)
+    data = synth.generate(w, DEV)
+    p = GtoPass(w, DEV)
+    p.build_tree(data["draft"])
+    weight = 2.0 / w.B
+    p.token_loss(data["draft"], data["target"], data["d2t"], weight)
+    assert p.status() == 0
+    d2t = None if data["d2t"] is None else data["d2t"].cpu().numpy()
+    loss = p.token_stats["loss"].cpu().numpy()
+    grad = p.grad_root.float().cpu().numpy().astype(np.float64)
+    rel = 2.0 ** -8 if w.dtype != "f32" else 1e-5
+    for b, (H, g) in enumerate(_token_loss_reference(w, data, d2t)):
+        assert abs(loss[b] - H) <= 1e-4 * max(1.0, abs(H)), (b, loss[b], H)
+        assert np.all(np.abs(grad[b] - weight * g) <= 2e-3 * weight + rel * np.abs(weight * g)), b
+
+
+def test_token_loss_with_an_injective_map_that_is_not_increasing(harness):
+    """Any injective map is accepted: one that is not in id order takes the gathering kernel."""
+    from paper_2509_22134_b200.runner import GtoPass
+    w = synth.Workload("tok", B=16, V_draft=2048, V_target=8200, D=2, k=4, g=8, dtype="bf16", seed=31)
+    data = synth.generate(w, DEV)
+    d2t = data["d2t"].clone()
+    d2t[100:1100] = data["d2t"][100:1100].flip(0)          # still injective
+    p = GtoPass(w, DEV)
+    p.build_tree(data["draft"])
+    p.token_loss(data["draft"], data["target"], d2t, 0.5)
+    assert p.status() == 0
+    loss = p.token_stats["loss"].cpu().numpy()
+    grad = p.grad_root.float().cpu().numpy().astype(np.float64)
+    for b, (H, g) in enumerate(_token_loss_reference(w, data, d2t.cpu().numpy())):
+        assert abs(loss[b] - H) <= 1e-4 * max(1.0, abs(H))
+        assert np.all(np.abs(grad[b] - 0.5 * g) <= 1e-3 + 2.0 ** -8 * np.abs(0.5 * g))
+
+
+@pytest.mark.parametrize("live_rows", [False, True])
+def test_token_loss_accumulates_into_the_surrogate_gradient(harness, live_rows):
+    """L = L_token + omega L_GTO (Sec. 3.2) in one buffer: slice [b, 0, :] holds the sum of the two
+    oracle gradients of the root row where the accepted path is live, the token gradient alone
+    elsewhere; the other slices are left as the surrogate call wrote them."""
+    from paper_2509_22134_b200 import binding as gto
+    w = synth.Workload("tok", B=32, V_draft=4104, V_target=9000, D=4, k=5, g=30, dtype="bf16",
+                       seed=33, grad_scale=0.5)
+    p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS if live_rows else 0)
+    if live_rows:
+        p.grad.fill_(9.0)                                    # the caller's garbage in dead rows
+        p.surrogate_grad(data["draft"])
+    if not live_rows:
+        harness.check_against_oracle(w, p, data, groups=list(range(w.B // w.m)))
+    before = p.grad.clone()
+    live = ((p.reward["path_len"] > 0) & (p.stats["coeff"] != 0)).cpu().numpy()
+    assert live.any() and (~live).any()
+    weight = 1.0 / w.B
+    p.token_loss_accumulate(data["draft"], data["target"], data["d2t"], weight)
+    assert p.status() == 0
+    assert torch.equal(p.grad[:, 1:], before[:, 1:])
+    d2t = data["d2t"].cpu().numpy()
+    got = p.grad[:, 0].float().cpu().numpy().astype(np.float64)
+    sur = before[:, 0].float().cpu().numpy().astype(np.float64)
+    loss = p.token_stats["loss"].cpu().numpy()
+    for b, (H, g) in enumerate(_token_loss_reference(w, data, d2t)):
+        want = weight * g + (sur[b] if live[b] else 0.0)
+        assert abs(loss[b] - H) <= 1e-4 * max(1.0, abs(H))
+        assert np.all(np.abs(got[b] - want) <= 2e-3 * (weight + w.grad_scale) + 2.0 ** -8 * np.abs(want)), b
 
 
 def test_reward_from_host_rows_copies_only_the_needed_rows(harness):
@@ -324,20 +431,31 @@ def test_nonfinite_row_sets_status_and_bad_args_are_refused(harness):
         gto.gto_create(cfg, 0)
 
 
-@pytest.mark.parametrize("cfg_id,groups", [(1, [0, 31, 63]), (2, [0, 127]), (3, [0, 63]), (4, [0, 255])])
-def test_baseline_configs_sampled_groups(harness, cfg_id, groups):
+@pytest.mark.parametrize("cfg_id", [1, 2, 3, 4])
+def test_baseline_configs_sampled_groups(harness, oracle_workers, cfg_id):
     """The full-size workloads in the launch configuration the benchmark times; the oracle
-    checks whole groups sampled from the ends of the batch."""
+    checks whole groups: the first, the last and eight more drawn over the whole batch, each on
+    its own host core."""
     w = synth.WORKLOADS[cfg_id]
     free, _ = torch.cuda.mem_get_info()
     need = (w.G * w.B * w.D * w.k * w.V_draft + w.G * w.B * w.R * w.V_target + w.B * w.D * w.V_draft) * 2
     if free < need * 1.1 + (4 << 30):
         pytest.skip("not enough free device memory for this workload")
     from paper_2509_22134_b200 import binding as gto
+    n_groups = w.B // w.m
+    rng = np.random.default_rng(900 + cfg_id)
+    groups = sorted({0, n_groups - 1} | {int(x) for x in rng.choice(n_groups, size=8, replace=False)})
     # workload 2 is the one the benchmark times: same flags as there
     p, data = harness.run_pass(w, DEV, flags=gto.GTO_FLAG_GRAD_LIVE_ROWS if cfg_id == 2 else 0)
-    rep = harness.check_against_oracle(w, p, data, groups=groups)
+    rep = harness.check_against_oracle(w, p, data, groups=groups, workers=oracle_workers)
+    assert rep["positions"] == len(groups) * w.m
     print(cfg_id, rep)
+    import json, os
+    out_dir = os.environ.get("GTO_PARITY_REPORT_DIR")      # optional record of the counts
+    if out_dir:
+        os.makedirs(out_dir, exist_ok=True)
+        with open(os.path.join(out_dir, f"parity_workload{cfg_id}.json"), "w") as f:
+            json.dump(dict(workload=w.name, groups=groups, **rep), f)
     # rows sampled over the whole batch, one by one against the oracle
     from oracle import gto_oracle as orc
     rng = np.random.default_rng(cfg_id)
