@@ -443,9 +443,14 @@ def run_gpu(args, w, rank, world, local_rank):
         tot, cnt = gto.gto_kernel_times(p.ctx)["token_loss"]
         gto.gto_kernel_timing(p.ctx, False)
         tok_bytes = w.B * 3 * w.V_draft * w.elem_bytes   # draft row, mapped target logits, gradient row
+        # what has to cross the memory bus: the mapped ids are spread over the whole target row
+        tok_streamed = w.B * (2 * w.V_draft + w.V_target) * w.elem_bytes
         extras["token_loss"] = {"ms": tot / cnt, "algorithmic_bytes": tok_bytes,
                                 "gbs": tok_bytes / (tot / cnt * 1e-3) / 1e9,
-                                "note": "Eq. 13 on the B root rows, timed alone (not part of the step)"}
+                                "streamed_bytes": tok_streamed,
+                                "streamed_gbs": tok_streamed / (tot / cnt * 1e-3) / 1e9,
+                                "note": "Eq. 13 on the B root rows, timed alone (not part of the step); "
+                                        "the span covers the call's launches (id-map bitmap, streaming kernel)"}
 
     # ---- (4) end to end: host buffers, copies inside the timed region
     e2e = run_e2e(args, w, dev, b0, world) if not args.no_e2e else None

@@ -19,7 +19,7 @@
  * the row list for gto_tree_reward_host) and keeps no caller pointer
  * after a call returns.  Calls enqueue work on `stream` (a cudaStream_t passed as void*)
  * and return without synchronising; argument errors are returned at once and launch
- * nothing.  Data faults (a non-finite row sum, a bounded wait that ran out) are recorded
+ * nothing.  Data faults (a non-finite row sum, an index out of range in a caller's table) are recorded
  * in a device status word read by gto_device_status.  A context is not thread-safe;
  * use one per host thread and device.  No entry point writes to stdout or throws.
  */
@@ -41,7 +41,7 @@ typedef enum {
   GTO_ERR_WORKSPACE = 3,   /* workspace allocation failed                                */
   GTO_ERR_CUDA = 4,        /* a CUDA runtime call failed                                 */
   GTO_ERR_NONFINITE = 5,   /* device status: a row's log-sum-exp was not finite          */
-  GTO_ERR_TIMEOUT = 6,     /* device status: a bounded wait inside a kernel ran out      */
+  /* 6 is not used: no kernel of the library waits on anything                            */
   GTO_ERR_TOO_LARGE = 7,   /* gto_build_tree_noalloc: batch exceeds the fixed scratch    */
   GTO_ERR_BAD_INDEX = 8    /* device status: an index in a caller's table (d2t, a tree's
                               rows, tokens or parents, a path's rows) was out of range; the
@@ -62,6 +62,10 @@ enum {
                                   for tests and tuning                                      */
   GTO_FLAG_SEQ_ALL_NODES = 8u, /* Eq. 5 over the root-to-node sequence of every selected node
                                   instead of the root-to-leaf sequences only                 */
+  GTO_FLAG_PATH_MAX_EXPECTED = 32u, /* the "longest accepted sequence" of Sec. 3.2 read as the
+                                  candidate sequence with the largest expected acceptance length
+                                  L_i of Eq. 3 (lowest list position on ties), reported whole, root
+                                  to its last node; default: the greedy-target verification walk */
   GTO_FLAG_GRAD_LIVE_ROWS = 4u /* gto_group_surrogate_grad writes only the rows that carry a
                                   gradient (j < path_len[b] and coeff[b] != 0) and leaves the
                                   rest of grad untouched, instead of filling it with zeros   */
@@ -248,7 +252,7 @@ gto_status gto_token_loss_accumulate(gto_ctx* ctx, const void* draft_logits,
 gto_status gto_sample_groups(int32_t s, int32_t m, int32_t K, const double* u, int32_t* starts);
 
 /* Synchronises `stream`, then reads and clears the device status word:
- * *host_code = GTO_OK, GTO_ERR_NONFINITE, GTO_ERR_BAD_INDEX or GTO_ERR_TIMEOUT.  Kernels check
+ * *host_code = GTO_OK, GTO_ERR_NONFINITE or GTO_ERR_BAD_INDEX.  Kernels check
  * every index they take from a caller's table before using it as an address. */
 gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code);
 

@@ -88,7 +88,8 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
     for i in range(n):
         d_i = np.asarray(draft[:, i], dtype=np.float64)
         t_i = np.asarray(target[:, i], dtype=np.float64)
-        f = orc.position_forward(d_i, t_i, D, k, g, d2t, cfg.eta, agg, getattr(cfg, "all_nodes", False))
+        f = orc.position_forward(d_i, t_i, D, k, g, d2t, cfg.eta, agg, getattr(cfg, "all_nodes", False),
+                                 getattr(cfg, "expected_path", False))
         fwd.append(f)
         for t in range(G):
             tr = f["trees"][t]
@@ -140,6 +141,16 @@ def check_positions(cfg, draft, target, d2t, gpu, old_logp_fn, positions):
         path = f["path"]
         l = len(path["nodes"])
         rep["mean_path_len"] += l / n
+        if getattr(cfg, "expected_path", False) and list(gpu["path_node"][i][:gpu["path_len"][i]]) != path["nodes"]:
+            # the arg-max over L is a floating-point decision: another sequence is excused only if
+            # its L is within the tie window of the best one
+            rw0 = f["rewards"][0]
+            other = int(gpu["path_node"][i][gpu["path_len"][i] - 1]) if gpu["path_len"][i] > 0 else -1
+            assert other in [int(x) for x in rw0["leaves"]] and \
+                rw0["Lc"][path["nodes"][-1]] - rw0["Lc"][other] < TIE_TOL, f"sequence choice at {positions[i]}"
+            rep["near_tie_trees"] += 1
+            excused[i] = True
+            continue
         assert gpu["path_len"][i] == l, f"path length {gpu['path_len'][i]} vs {l} at {positions[i]}"
         assert list(gpu["path_node"][i][:l]) == path["nodes"]
         assert list(gpu["path_row"][i][:l]) == path["rows"]

@@ -14,6 +14,7 @@ Steps and the passages they follow:
   target_node_probs     Sec. 3.1, the factor T(x_{t+k} | ...) of Eq. 4
   tree_reward           Sec. 3.1 Eq. 3-5 (expected acceptance length, smooth max)
   longest_accepted      Sec. 3.2 "longest accepted sequence", App. A case (b) (greedy target)
+  most_expected_sequence  the other reading of that phrase: the sequence with the largest L_i
   group_advantages      Sec. 3.2 Eq. 9-10 (debias, standardise)
   clipped_surrogate     Sec. 3.2 Eq. 11-12 (length-normalised ratio, PPO clip)
   surrogate_grad_rows   derivative of Eq. 12 with respect to the draft logits
@@ -303,6 +304,27 @@ def longest_accepted(tree, target, d2t=None):
     return dict(nodes=nodes, rows=rows, tokens=toks, logp=lps)
 
 
+def most_expected_sequence(tree, Lc, leaves):
+    """The other reading of "longest accepted sequence" (Sec. 3.2): instead of verifying
+    greedily, take the candidate sequence S_i whose expected acceptance length L_i (Eq. 3) is
+    the largest - the lowest list position on ties - and return it whole, root to its last
+    node, in the form longest_accepted uses.  Lc, leaves: from tree_reward.
+    """
+    leaves = [int(n) for n in leaves]
+    best = leaves[0]
+    for n in leaves[1:]:
+        if Lc[n] > Lc[best]:
+            best = n
+    chain = []
+    n = best
+    while n >= 0:
+        chain.append(n)
+        n = int(tree.parent[n])
+    chain.reverse()
+    return dict(nodes=chain, rows=[int(tree.ctx_row[n]) for n in chain],
+                tokens=[int(tree.token[n]) for n in chain], logp=[float(tree.logp[n]) for n in chain])
+
+
 # --------------------------------------------------------------------------- O8
 def group_advantages(r_cur, r_ref, m, delta=1e-6, unbiased=False, debias=True):
     """Eq. 9: R_i = r(T_i) - r(T_i under the reference draft); Eq. 10: standardise R
@@ -376,11 +398,13 @@ def surrogate_grad_rows(draft_rows, row_lse, tokens, coeff, D, V):
 
 
 # ------------------------------------------------------------------ whole passes
-def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE, all_nodes=False):
+def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE, all_nodes=False,
+                     expected_path=False):
     """Trees, rewards and the longest accepted sequence of one position.
 
     draft_b: [G, D, k, V_d], target_b: [G, R, V_t] with G = 2 (0 = current draft,
-    1 = frozen reference draft).  Returns dict(trees, probs, rewards, path).
+    1 = frozen reference draft).  expected_path selects most_expected_sequence instead of the
+    greedy walk.  Returns dict(trees, probs, rewards, path).
     """
     G = draft_b.shape[0]
     trees, probs, rewards = [], [], []
@@ -393,12 +417,16 @@ def position_forward(draft_b, target_b, D, k, g, d2t=None, eta=1.0, agg=AGG_LSE,
         trees.append(tree)
         probs.append(p)
         rewards.append(rw)
-    path = longest_accepted(trees[0], target_b[0], d2t)
+    if expected_path:
+        path = most_expected_sequence(trees[0], rewards[0]["Lc"], rewards[0]["leaves"])
+    else:
+        path = longest_accepted(trees[0], target_b[0], d2t)
     return dict(trees=trees, rewards=rewards, path=path)
 
 
 def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, agg=AGG_LSE,
-               delta=1e-6, eps=0.2, grad_scale=1.0, unbiased=False, debias=True, all_nodes=False):
+               delta=1e-6, eps=0.2, grad_scale=1.0, unbiased=False, debias=True, all_nodes=False,
+               expected_path=False):
     """The whole pass of Algorithm 1's inner loop on ONE group of m positions: trees and
     rewards of both drafts, the longest accepted sequences, Eq. 9-12 and the gradient rows.
     Sequences the functions above; adds no arithmetic of its own.
@@ -411,7 +439,7 @@ def group_pass(draft_g, target_g, D, k, g, m, old_logp_fn, d2t=None, eta=1.0, ag
     V = draft_g.shape[-1]
     fwd = [position_forward(np.asarray(draft_g[:, i], dtype=np.float64),
                             np.asarray(target_g[:, i], dtype=np.float64), D, k, g, d2t, eta, agg,
-                            all_nodes)
+                            all_nodes, expected_path)
            for i in range(m)]
     r_cur = np.array([f["rewards"][0]["r"] for f in fwd])
     r_ref = np.array([f["rewards"][1]["r"] for f in fwd])

@@ -20,6 +20,7 @@ GTO_F32, GTO_BF16, GTO_F16 = 0, 1, 2
 GTO_AGG_LSE, GTO_AGG_MAX, GTO_AGG_MEAN = 0, 1, 2
 GTO_FLAG_STD_UNBIASED, GTO_FLAG_NO_DEBIAS, GTO_FLAG_GRAD_LIVE_ROWS, GTO_FLAG_SEQ_ALL_NODES = 1, 2, 4, 8
 GTO_FLAG_FORCE_ROW_SPLIT = 16
+GTO_FLAG_PATH_MAX_EXPECTED = 32
 
 if not os.path.exists(LIB_PATH):
     raise RuntimeError(

@@ -120,7 +120,6 @@ const char* gto_status_string(gto_status s) {
     case GTO_ERR_WORKSPACE: return "workspace allocation failed";
     case GTO_ERR_CUDA: return "CUDA runtime error";
     case GTO_ERR_NONFINITE: return "non-finite logit row";
-    case GTO_ERR_TIMEOUT: return "bounded device wait ran out";
     case GTO_ERR_TOO_LARGE: return "batch exceeds the fixed scratch of the no-allocation call";
     case GTO_ERR_BAD_INDEX: return "an index in a caller's table was out of range";
   }
@@ -495,8 +494,7 @@ gto_status gto_device_status(gto_ctx* ctx, void* stream, int32_t* host_code) {
       cudaMemsetAsync(ctx->status, 0, sizeof(word), s) != cudaSuccess ||
       cudaStreamSynchronize(s) != cudaSuccess)
     return GTO_ERR_CUDA;
-  *host_code = (word & gto::kStatusTimeout)     ? GTO_ERR_TIMEOUT
-               : (word & gto::kStatusBadIndex)  ? GTO_ERR_BAD_INDEX
+  *host_code = (word & gto::kStatusBadIndex)    ? GTO_ERR_BAD_INDEX
                : (word & gto::kStatusNonFinite) ? GTO_ERR_NONFINITE
                                                 : GTO_OK;
   return GTO_OK;

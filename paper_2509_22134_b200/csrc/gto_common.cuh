@@ -13,7 +13,6 @@ constexpr unsigned kFull = 0xffffffffu;
 
 // bits of the device status word
 constexpr int kStatusNonFinite = 1;
-constexpr int kStatusTimeout = 2;
 constexpr int kStatusBadIndex = 4;  // an index read from a caller's table was out of range
 
 constexpr float kLog2e = 1.4426950408889634f;

@@ -45,30 +45,33 @@ __device__ __forceinline__ double warp_sum_f64(double v) {
 }
 
 // ------------------------------------------------------------------ bitmap of the id map
-// map_state[0] = 1 if the map is not strictly increasing, map_state[1] = set bits counted.
-__global__ void token_map_mark_kernel(const int32_t* __restrict__ d2t, int V_draft, int V_target,
-                                      uint32_t* __restrict__ bitmap, int32_t* __restrict__ map_state,
-                                      int32_t* __restrict__ status) {
-  const int v = blockIdx.x * blockDim.x + threadIdx.x;
-  if (v >= V_draft) return;
-  const int id = d2t[v];
-  if (id < 0 || id >= V_target) {
-    atomicOr(status, kStatusBadIndex);
-    atomicOr(map_state, 1);  // ranks would no longer be draft ids: leave it to the gathering kernel
-    return;
-  }
-  if (v > 0 && d2t[v - 1] >= id) atomicOr(map_state, 1);
-  atomicOr(bitmap + (id >> 5), 1u << (id & 31));
-}
-
-// prefix[w] = number of mapped target ids below 32 w (one CTA; a few thousand words).
-__global__ void __launch_bounds__(1024) token_map_scan_kernel(const uint32_t* __restrict__ bitmap,
-                                                             int n_words,
-                                                             uint32_t* __restrict__ prefix) {
+// One CTA builds, for the call's id map: bitmap[w] bit i = target id 32 w + i is the image of a
+// draft id; prefix[w] = number of mapped target ids below 32 w; map_state[0] = 1 if the map is
+// not strictly increasing or holds an id outside the target vocabulary (the streaming kernel
+// then leaves the call to the gathering kernel).  A few thousand words: one launch is cheaper
+// than a grid-wide version with its extra launches.
+__global__ void __launch_bounds__(1024) token_map_build_kernel(
+    const int32_t* __restrict__ d2t, int V_draft, int V_target, int n_words, uint32_t* bitmap,
+    uint32_t* __restrict__ prefix, int32_t* map_state, int32_t* __restrict__ status) {
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t carry;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) carry = 0;
+  for (int w = tid; w < n_words; w += 1024) bitmap[w] = 0;
+  if (tid == 0) {
+    carry = 0;
+    map_state[0] = 0;
+  }
+  __syncthreads();
+  for (int v = tid; v < V_draft; v += 1024) {
+    const int id = d2t[v];
+    if (id < 0 || id >= V_target) {
+      atomicOr(status, kStatusBadIndex);
+      atomicOr(map_state, 1);  // ranks would no longer be draft ids
+      continue;
+    }
+    if (v > 0 && d2t[v - 1] >= id) atomicOr(map_state, 1);
+    atomicOr(bitmap + (id >> 5), 1u << (id & 31));
+  }
   __syncthreads();
   for (int base = 0; base < n_words; base += 1024) {
     const int w = base + tid;
@@ -123,28 +126,24 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
   using Elem = typename T::Storage;
   Elem* s_t = reinterpret_cast<Elem*>(s_raw);
 
-  // ---- pass A: the range's mapped target logits into shared memory; running max and sum
+  // ---- pass A: the range's mapped target logits into shared memory, then their max and sum
   float m = -INFINITY, s = 0.f;
-  auto take = [&](const float (&t)[E], unsigned keep) {
-    float vmax = -INFINITY;
+  auto take = [&](const float (&t)[E]) {
+    float vmax = t[0];
 #pragma unroll
-    for (int e = 0; e < E; ++e)
-      if (keep >> e & 1) vmax = fmaxf(vmax, t[e]);
+    for (int e = 1; e < E; ++e) vmax = fmaxf(vmax, t[e]);
     if (vmax > m) {
       s *= ex2_approx((m - vmax) * kLog2e);
       m = vmax;
     }
+    if (m != -INFINITY) {
 #pragma unroll
-    for (int e = 0; e < E; ++e)
-      if (keep >> e & 1) s += ex2_approx((t[e] - m) * kLog2e);
+      for (int e = 0; e < E; ++e) s += ex2_approx((t[e] - m) * kLog2e);
+    }
   };
   if (a.d2t == nullptr) {
     for (int i = vec0 + tid; i < vec1; i += kTokThreads) {
-      const uint4 v = ld_stream16(zt + static_cast<size_t>(i) * 16);
-      reinterpret_cast<uint4*>(s_raw)[i - vec0] = v;
-      float t[E];
-      T::unpack(v, t);
-      take(t, (1u << E) - 1u);
+      reinterpret_cast<uint4*>(s_raw)[i - vec0] = ld_stream16(zt + static_cast<size_t>(i) * 16);
     }
   } else if (id1 > id0) {
     const int t_lo = a.d2t[id0], t_hi = a.d2t[id1 - 1];  // target ids of the range's ends
@@ -170,24 +169,24 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
         // of the first mapped one among them
         const int first = (i0 + u * kTokThreads) * E;
         const unsigned bits = (word[u] >> (first & 31)) & ((1u << E) - 1u);
-        if (bits == 0) continue;
+        unsigned todo = bits;
         int rank = static_cast<int>(pre[u]) + __popc(word[u] & ((1u << (first & 31)) - 1u));
-        float t[E];
-        T::unpack(v[u], t);
-        unsigned keep = 0;
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-          if (bits >> e & 1) {
-            if (rank >= id0 && rank < id1) {  // neighbouring ranges share their end vectors
-              s_t[rank - id0] = T::element(v[u], e);
-              keep |= 1u << e;
-            }
-            ++rank;
-          }
+        while (todo) {  // about E * V_draft / V_target mapped ids per vector
+          const int e = __ffs(todo) - 1;
+          todo &= todo - 1;
+          // neighbouring ranges share their end vectors: keep the ids of this range only
+          if (rank >= id0 && rank < id1) s_t[rank - id0] = T::element(v[u], e);
+          ++rank;
         }
-        take(t, keep);
       }
     }
+  }
+  __syncthreads();
+  // the range's log-sum-exp from shared memory (dense, in draft-id order)
+  for (int i = tid; i < vec1 - vec0; i += kTokThreads) {
+    float t[E];
+    T::unpack(reinterpret_cast<const uint4*>(s_raw)[i], t);
+    take(t);
   }
   {
     const float wm = warp_max_f32(m);
@@ -429,37 +428,34 @@ cudaError_t launch_stream(const TokenLossArgs& a, int C, size_t smem, cudaStream
 
 }  // namespace
 
-// CTAs per position for the streaming kernel: enough that a CTA's share of the row fits in
-// shared memory (at most 64 KB, so that several CTAs stay resident per SM) and that a small
-// batch still fills the device; 0 = the row is too long for a portable cluster.
-int token_loss_cluster_size(int B, int V_draft, int dtype, int sms) {
+// CTAs per position for the streaming kernel, from timings on B200 (us per call, B = 1024,
+// bf16): with an id map 32 000 -> 128 256, 2 CTAs per position are fastest; without a map the
+// gathering kernel (target re-read from L2) wins while a row is short (54 vs 67 at 32 000 ids)
+// and 4 CTAs win on long rows (155 vs 179 at 151 936 ids).  Small batches take the largest
+// portable cluster so that the device fills.  0 = use the gathering kernel.
+int token_loss_cluster_size(int B, int V_draft, bool mapped, int dtype, int sms) {
 #ifdef GTO_TOK_CLUSTER
   return GTO_TOK_CLUSTER;  // tuning builds
 #endif
   const size_t row = static_cast<size_t>(V_draft) * elem_bytes(dtype);
-  for (int C = 1; C <= 8; C *= 2) {
-    const bool fits = (row + C - 1) / C + 64 <= 64 * 1024;
-    const bool fills = static_cast<int64_t>(B) * C >= 4ll * sms || C == 8;
-    if (fits && fills) return C;
-  }
-  return 0;
+  if (!mapped && row < 128 * 1024 && B >= sms) return 0;
+  int C = mapped ? 2 : 4;
+  while (C < 8 && static_cast<int64_t>(B) * C < 2ll * sms) C *= 2;  // a small batch
+  while (C < 8 && (row + C - 1) / C + 64 > 96 * 1024) C *= 2;        // a CTA's share must fit
+  return (row + C - 1) / C + 64 <= 200 * 1024 ? C : 0;
 }
 
 cudaError_t launch_token_loss(const TokenLossArgs& a, int sms, cudaStream_t stream,
                               int64_t* launches) {
   if (a.B <= 0) return cudaSuccess;
-  const int C = token_loss_cluster_size(a.B, a.V_draft, a.dtype, sms);
+  const int C = token_loss_cluster_size(a.B, a.V_draft, a.d2t != nullptr, a.dtype, sms);
   cudaError_t e = cudaSuccess;
   if (C > 0 && a.d2t != nullptr) {
     // the bitmap of the map's image and its prefix counts
     const int n_words = (a.V_target + 31) / 32 + 1;
-    e = cudaMemsetAsync(a.map_bits, 0, static_cast<size_t>(n_words) * 4, stream);
-    if (e == cudaSuccess) e = cudaMemsetAsync(a.map_state, 0, 8, stream);
-    if (e != cudaSuccess) return e;
-    token_map_mark_kernel<<<(a.V_draft + 255) / 256, 256, 0, stream>>>(
-        a.d2t, a.V_draft, a.V_target, a.map_bits, a.map_state, a.status);
-    token_map_scan_kernel<<<1, 1024, 0, stream>>>(a.map_bits, n_words, a.map_prefix);
-    *launches += 2;
+    token_map_build_kernel<<<1, 1024, 0, stream>>>(a.d2t, a.V_draft, a.V_target, n_words, a.map_bits,
+                                                   a.map_prefix, a.map_state, a.status);
+    ++*launches;
   }
   if (C > 0) {
     const int E = 16 / elem_bytes(a.dtype);

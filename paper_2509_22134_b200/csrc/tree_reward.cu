@@ -170,7 +170,41 @@ __global__ void __launch_bounds__(kWarpsPerCta * 32) tree_reward_kernel(RewardAr
 
   // ---- longest accepted sequence of the current draft's tree (t = 0): follow the greedy
   //      target token through the selected children
-  if (tree < a.B) {
+  if (tree < a.B && (a.flags & GTO_FLAG_PATH_MAX_EXPECTED)) {
+    // the other reading: the sequence with the largest L (Eq. 3), lowest list position on
+    // ties, taken whole from the root to its last node
+    const int b = tree;
+    double best = -INFINITY;
+    int at = g;
+    for (int n = lane; n < g; n += 32)
+      if ((all_nodes || !sm.has_child[n]) && sm.Lc[n] > best) {
+        best = sm.Lc[n];
+        at = n;
+      }
+    const double top = warp_max_f64(best);
+    at = __reduce_min_sync(kFull, best == top ? at : g);
+    int len = 0;
+    if (at < g) {
+      len = sm.depth[at];
+      int n = at;
+      for (int j = len - 1; j >= 0 && n >= 0; --j) {  // every lane walks the same chain
+        if (lane == 0) {
+          a.out.path_node[b * D + j] = n;
+          a.out.path_row[b * D + j] = a.tree.node_ctx_row[nb + n];
+          a.out.path_token[b * D + j] = a.tree.node_token[nb + n];
+          a.out.path_logp[b * D + j] = a.tree.node_logp[nb + n];
+        }
+        n = sm.parent[n];
+      }
+    }
+    if (lane == 0) a.out.path_len[b] = len;
+    for (int j = len + lane; j < D; j += 32) {
+      a.out.path_node[b * D + j] = -1;
+      a.out.path_row[b * D + j] = -1;
+      a.out.path_token[b * D + j] = -1;
+      a.out.path_logp[b * D + j] = 0.f;
+    }
+  } else if (tree < a.B) {
     const int b = tree;
     int cur = -1, row = 0, len = 0;
     while (len < D) {

@@ -272,3 +272,59 @@ def test_all_nodes_variant_sums_over_every_root_to_node_sequence():
     assert got["r"] >= orc.tree_reward(tree, p, eta=1.3)["r"]     # a superset of sequences
     assert orc.tree_reward(tree, p, agg=orc.AGG_MAX, all_nodes=True)["r"] == \
         orc.tree_reward(tree, p, agg=orc.AGG_MAX)["r"]            # the longest paths end in leaves
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_most_expected_sequence_extends_the_greedy_path_for_one_hot_targets(seed):
+    """App. A case (b): with one-hot target rows L_i is the length of the prefix S_i shares with
+    the greedy target trajectory, so a sequence of largest L_i starts with the whole greedy
+    accepted path and its L equals the accepted length."""
+    rng = np.random.default_rng(80 + seed)
+    D, k, g, V = 4, 3, 14, 8
+    draft = rng.normal(size=(D, k, V)) * 2
+    tree = orc.build_tree(draft, D, k, g)
+    R = 1 + (D - 1) * k
+    greedy = np.array([int(np.argsort(-draft[orc.draft_slot_of_row(r, k)])[rng.integers(0, 2)]) for r in range(R)])
+    target = np.full((R, V), -1000.0)
+    target[np.arange(R), greedy] = 1000.0
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    walk = orc.longest_accepted(tree, target)
+    best = orc.most_expected_sequence(tree, rw["Lc"], rw["leaves"])
+    l = len(walk["nodes"])
+    assert best["nodes"][:l] == walk["nodes"] and best["rows"][:l] == walk["rows"]
+    assert rw["Lc"][best["nodes"][-1]] == pytest.approx(l, abs=1e-12)
+    assert best["nodes"][-1] in rw["leaves"]
+    # parent-linked from the root, one node per depth
+    assert [int(tree.depth[n]) for n in best["nodes"]] == list(range(1, len(best["nodes"]) + 1))
+    assert all(tree.parent[b] == a for a, b in zip(best["nodes"], best["nodes"][1:]))
+    assert tree.parent[best["nodes"][0]] == -1
+
+
+def test_most_expected_sequence_is_the_argmax_of_explicit_path_sums():
+    """Independent restatement: every leaf's L by explicit products along its path; the first
+    leaf of largest L wins; tokens, rows and log-probabilities are those of its path."""
+    draft, target, tree = tiny_case(11, V=6, D=4, k=3, g=12)
+    p, _ = orc.target_node_probs(tree, target)
+    rw = orc.tree_reward(tree, p)
+    chains = {}
+    for n in rw["leaves"]:
+        chain, x = [], int(n)
+        while x >= 0:
+            chain.append(x)
+            x = int(tree.parent[x])
+        chains[int(n)] = chain[::-1]
+    L = {n: sum(np.prod([p[a] for a in c[:j + 1]]) for j in range(len(c))) for n, c in chains.items()}
+    want = max(sorted(L), key=lambda n: (L[n], -n))
+    got = orc.most_expected_sequence(tree, rw["Lc"], rw["leaves"])
+    assert got["nodes"] == chains[want]
+    assert got["tokens"] == [int(tree.token[n]) for n in chains[want]]
+    assert got["rows"] == [int(tree.ctx_row[n]) for n in chains[want]]
+    assert got["logp"] == [float(tree.logp[n]) for n in chains[want]]
+    # not simply the deepest or the first leaf
+    assert len({len(c) for c in chains.values()}) > 1
+    # an exact tie goes to the lower list position
+    Lc = rw["Lc"].copy()
+    a, b = sorted(chains)[:2]
+    Lc[a] = Lc[b] = Lc.max() + 1.0
+    assert orc.most_expected_sequence(tree, Lc, rw["leaves"])["nodes"][-1] == a

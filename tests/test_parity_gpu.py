@@ -121,6 +121,20 @@ def test_variants_max_mean_unbiased_nodebias(harness):
     harness.check_against_oracle(w4, p, data, groups=[0, 1], cfg_extra=dict(all_nodes=True))
 
 
+@pytest.mark.parametrize("all_nodes", [False, True])
+def test_path_as_the_sequence_of_largest_expected_length(harness, all_nodes):
+    """The flagged reading of "longest accepted sequence": arg-max of L_i (Eq. 3) over the
+    tree's sequences, root to last node; the surrogate and its gradient then run on that path."""
+    from paper_2509_22134_b200 import binding as gto
+    w = synth.Workload("lpath", B=32, V_draft=4104, V_target=9000, D=5, k=6, g=40, seed=707)
+    flags = gto.GTO_FLAG_PATH_MAX_EXPECTED | (gto.GTO_FLAG_SEQ_ALL_NODES if all_nodes else 0)
+    p, data = harness.run_pass(w, DEV, flags=flags)
+    rep = harness.check_against_oracle(w, p, data, groups=list(range(w.B // w.m)),
+                                       cfg_extra=dict(expected_path=True, all_nodes=all_nodes))
+    assert int(p.reward["path_len"].min()) >= 1          # a tree always has a best sequence
+    print(rep)
+
+
 @pytest.mark.parametrize("grad_scale", [1.0, 0.5 / 16])
 @pytest.mark.parametrize("std_delta", [1e-6, 1e-2])
 @pytest.mark.parametrize("clip_eps", [0.05, 0.2, 0.5])

@@ -219,3 +219,13 @@ def test_pass_that_hands_the_advantages_to_the_wrong_positions(monkeypatch):
     monkeypatch.setattr(orc, "group_advantages", mutant)
     # (finite differences cannot see this one: loss and gradient would use the same wrong values)
     assert fails(tp.test_hand_worked_group_rows_tokens_and_advantages_land_where_they_belong)
+
+
+def test_expected_path_that_takes_the_deepest_leaf(monkeypatch):
+    real = orc.most_expected_sequence
+
+    def mutant(tree, Lc, leaves):
+        return real(tree, np.asarray(tree.depth, dtype=np.float64), leaves)   # ranks leaves by depth
+    monkeypatch.setattr(orc, "most_expected_sequence", mutant)
+    assert fails(tr.test_most_expected_sequence_is_the_argmax_of_explicit_path_sums) or \
+        any(fails(tr.test_most_expected_sequence_extends_the_greedy_path_for_one_hot_targets, s) for s in range(6))

@@ -28,6 +28,20 @@ def _trees_equal(a, b):
         assert torch.allclose(a[name].double(), b[name].double(), rtol=0, atol=1e-6), name
 
 
+def _matches_the_oracle(w, data, tree, positions):
+    """The no-allocation call's own output against the oracle's tree, node by node."""
+    import numpy as np
+    from oracle import gto_oracle as orc
+    for b in positions:
+        for t in range(w.G):
+            want = orc.build_tree(data["draft"][t, b].float().cpu().numpy().astype(np.float64), w.D, w.k, w.g)
+            for name, attr in (("node_token", "token"), ("node_parent", "parent"), ("node_depth", "depth"),
+                               ("node_ctx_row", "ctx_row"), ("node_slot", "slot"), ("node_pool", "pool")):
+                assert np.array_equal(tree[name][t, b].cpu().numpy(), getattr(want, attr)), (name, t, b)
+            assert np.max(np.abs(tree["node_score"][t, b].cpu().numpy() - want.score)) <= 1e-5
+            assert np.max(np.abs(tree["row_lse"][t, b].cpu().numpy() - want.row_lse)) <= 2e-6
+
+
 def test_two_calls_in_a_row_match_the_context_call():
     from paper_2509_22134_b200 import binding as gto
     # two different shapes back to back, the larger first, so stale scratch would show
@@ -48,6 +62,7 @@ def test_two_calls_in_a_row_match_the_context_call():
         torch.cuda.synchronize()
         _trees_equal(got, want)
         gto.gto_destroy(ctx)
+        _matches_the_oracle(w, data, got, positions=(0, w.B - 1))
 
 
 def test_a_batch_beyond_the_fixed_scratch_is_refused():
