@@ -407,10 +407,18 @@ __global__ void __launch_bounds__(kTokThreads, 8) token_loss_gather_kernel(Token
 
 template <typename T>
 cudaError_t launch_stream(const TokenLossArgs& a, int C, size_t smem, cudaStream_t stream) {
-  cudaError_t e = cudaFuncSetAttribute(token_loss_stream_kernel<T>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  // raise the kernel's dynamic shared memory limit when a call needs more than any before it
+  // (per device: the attribute belongs to the device's copy of the function)
+  static int allowed[64] = {};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || static_cast<int>(smem) > allowed[dev]) {
+    e = cudaFuncSetAttribute(token_loss_stream_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) allowed[dev] = static_cast<int>(smem);
+  }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(a.B) * C);
   cfg.blockDim = dim3(kTokThreads);
