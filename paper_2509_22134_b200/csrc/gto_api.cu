@@ -24,6 +24,8 @@ struct gto_ctx {
   uint32_t* map_bits;   // token loss: bitmap of the id map's image, and
   uint32_t* map_prefix; //   the number of mapped ids below each of its words
   int32_t* map_state;   //   [0] = 1 if the map is not increasing
+  int32_t* live_list;   // gradient: slices that carry a gradient (GTO_FLAG_GRAD_LIVE_ROWS)
+  int32_t* live_count;
   int sms;
   int32_t* h_list;    // page-locked host copy of the work list: [0] = count, then the rows
   int64_t last_host_rows;
@@ -182,9 +184,11 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   const size_t map_words = static_cast<size_t>(c->V_target + 31) / 32 + 1;
   const size_t o_bits = off; off += align_up(map_words * sizeof(uint32_t));
   const size_t o_pre = off; off += align_up(map_words * sizeof(uint32_t));
+  const size_t o_live = off; off += align_up(static_cast<size_t>(c->B) * c->D * sizeof(int32_t));
   const size_t o_cnt = off; off += 256;
   const size_t o_st = off;  off += 256;
   const size_t o_ms = off;  off += 256;
+  const size_t o_lc = off;  off += 256;
   if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
     cudaGetLastError();
     delete ctx;
@@ -198,7 +202,9 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->map_bits = reinterpret_cast<uint32_t*>(ctx->ws + o_bits);
   ctx->map_prefix = reinterpret_cast<uint32_t*>(ctx->ws + o_pre);
   ctx->map_state = reinterpret_cast<int32_t*>(ctx->ws + o_ms);
-  if (cudaMemset(ctx->ws + o_cnt, 0, 768) != cudaSuccess ||
+  ctx->live_list = reinterpret_cast<int32_t*>(ctx->ws + o_live);
+  ctx->live_count = reinterpret_cast<int32_t*>(ctx->ws + o_lc);
+  if (cudaMemset(ctx->ws + o_cnt, 0, 1024) != cudaSuccess ||
       cudaMallocHost(&ctx->h_list, (rows + 1) * sizeof(int32_t)) != cudaSuccess) {
     cudaGetLastError();
     cudaFree(ctx->ws);
@@ -397,6 +403,11 @@ gto_status gto_group_surrogate_grad(gto_ctx* ctx, const void* draft, const gto_t
   a.grad = grad;
   a.out = *out;
   a.status = ctx->status;
+  if (c.flags & GTO_FLAG_GRAD_LIVE_ROWS) {
+    a.live_list = ctx->live_list;
+    a.live_count = ctx->live_count;
+    a.live_grid = ctx->sms * 8;
+  }
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   {
     LaunchSpan span(ctx, GTO_K_GROUP_STATS, s);

@@ -79,6 +79,9 @@ struct GradArgs {
   void* grad;
   gto_grad_stats out;
   int32_t* status;
+  int32_t* live_list;   // with GTO_FLAG_GRAD_LIVE_ROWS: workspace [B*D], the slices b*D + j that
+  int32_t* live_count;  //   carry a gradient and their number; null otherwise
+  int live_grid;        // CTAs that walk the list
 };
 struct TokenLossArgs {
   int B, k, R, V_draft, V_target, dtype;

@@ -66,8 +66,15 @@ __global__ void __launch_bounds__(kStatWarps * 32) group_stats_kernel(GradArgs a
     a.out.adv[b] = A;
     a.out.ratio[b] = s;
     a.out.active[b] = active ? 1 : 0;
-    a.out.coeff[b] =
+    const double coeff =
         active ? static_cast<double>(a.grad_scale) * (-1.0 / m) * A * s / lden : 0.0;
+    a.out.coeff[b] = coeff;
+    // the rows that carry a gradient, for the list-walking gradient kernel (the same test
+    // as there: the coefficient as fp32)
+    if (a.live_list != nullptr && static_cast<float>(coeff) != 0.f && l > 0) {
+      const int at = atomicAdd(a.live_count, l);
+      for (int j = 0; j < l; ++j) a.live_list[at + j] = b * D + j;
+    }
   }
   loss = wsum(loss);
   if (lane == 0) a.out.loss[grp] = loss;
@@ -123,16 +130,87 @@ __global__ void __launch_bounds__(kGradThreads) grad_rows_kernel(GradArgs a) {
   }
 }
 
+// The same rows from the list group_stats_kernel made: a bounded grid walks (row, quarter of
+// the row) units, so no CTA is launched for the ~93 % of the slices that carry no gradient.
+constexpr int kLiveParts = 4;
+
+template <typename T>
+__global__ void __launch_bounds__(kGradThreads) grad_live_rows_kernel(GradArgs a) {
+  constexpr int E = T::kPerVec;
+  constexpr int U = 4;  // vectors in flight per thread
+  const int nvec = a.V / E;
+  const int per = (nvec + kLiveParts - 1) / kLiveParts;
+  const int units = *a.live_count * kLiveParts;
+  for (int unit = blockIdx.x; unit < units; unit += gridDim.x) {
+    const int bj = a.live_list[unit / kLiveParts];
+    const int part = unit % kLiveParts;
+    const int b = bj / a.D;
+    const int row = a.reward.path_row[bj];
+    const int tok = a.reward.path_token[bj];
+    if (row < 0 || row >= a.R) {  // not a context row: report, write nothing from it
+      if (threadIdx.x == 0) atomicOr(a.status, kStatusBadIndex);
+      continue;
+    }
+    const float c = static_cast<float>(a.out.coeff[b]);
+    const float nref =
+        -static_cast<float>(a.row_lse[static_cast<size_t>(b) * a.R + row] * 1.4426950408889634);
+    const char* in = static_cast<const char*>(a.draft) +
+                     tensor_row(b, row, a.R, a.k - 1) * a.V * T::kBytes;
+    char* out = static_cast<char*>(a.grad) + static_cast<size_t>(bj) * a.V * T::kBytes;
+    const int v1 = min(nvec, (part + 1) * per);
+    for (int i0 = part * per + threadIdx.x; i0 < v1; i0 += U * kGradThreads) {
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * kGradThreads;
+        if (i < v1) v[u] = ld_stream16(in + static_cast<size_t>(i) * 16);
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * kGradThreads;
+        if (i >= v1) break;
+        float f[E];
+        T::unpack(v[u], f);
+#pragma unroll
+        for (int e = 0; e < E; ++e) f[e] = -c * ex2_approx(fmaf(f[e], kLog2e, nref));
+        const int rel = tok - i * E;
+        if (rel >= 0 && rel < E) {
+#pragma unroll
+          for (int e = 0; e < E; ++e)
+            if (e == rel) f[e] += c;
+        }
+        st_stream16(out + static_cast<size_t>(i) * 16, T::pack(f));
+      }
+    }
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_group_stats(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
   int groups = a.B / a.m;
+  if (a.live_list != nullptr) {
+    cudaError_t e = cudaMemsetAsync(a.live_count, 0, sizeof(int32_t), stream);
+    if (e != cudaSuccess) return e;
+  }
   group_stats_kernel<<<(groups + kStatWarps - 1) / kStatWarps, kStatWarps * 32, 0, stream>>>(a);
   ++*launches;
   return cudaGetLastError();
 }
 
 cudaError_t launch_grad_rows(const GradArgs& a, cudaStream_t stream, int64_t* launches) {
+  if (a.live_list != nullptr) {
+    // live rows only: a few waves of CTAs walk the list
+    const dim3 grid(a.live_grid), block(kGradThreads);
+    if (a.dtype == GTO_BF16)
+      grad_live_rows_kernel<Bf16><<<grid, block, 0, stream>>>(a);
+    else if (a.dtype == GTO_F16)
+      grad_live_rows_kernel<F16><<<grid, block, 0, stream>>>(a);
+    else
+      grad_live_rows_kernel<F32><<<grid, block, 0, stream>>>(a);
+    ++*launches;
+    return cudaGetLastError();
+  }
   int vec_per_row = a.V / (16 / elem_bytes(a.dtype));
   int split = (vec_per_row + kGradThreads * 8 - 1) / (kGradThreads * 8);  // ~8 vectors/thread
   if (split < 1) split = 1;

@@ -93,7 +93,9 @@ __device__ __forceinline__ int bits_below(const unsigned (&m)[kMaskWords], int q
 }
 
 template <int K>  // top-k known at compile time, or 0
-__global__ void __launch_bounds__(kTreeThreads) tree_build_kernel(TreeBuildArgs a) {
+// 16 resident CTAs per SM (32 registers, no spills): the 2048 trees of the paper's batch are then
+// resident at once instead of in two waves of a latency-bound kernel.
+__global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildArgs a) {
   extern __shared__ __align__(16) unsigned char dyn[];
   __shared__ TreeSmem sm;
   const int tid = threadIdx.x;
