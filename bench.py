@@ -452,8 +452,8 @@ def run_gpu(args, w, rank, world, local_rank):
                                 "streamed_bytes": tok_streamed,
                                 "streamed_gbs": tok_streamed / (tot / cnt * 1e-3) / 1e9,
                                 "note": "Eq. 13 on the B root rows, timed alone (not part of the step): "
-                                        "back-to-back calls between two events, so the figure includes the "
-                                        "call's small launches (id-map bitmap) and any host-side gap"}
+                                        "back-to-back calls between two events (one launch per call), so the "
+                                        "figure includes any host-side gap"}
 
     # ---- (4) end to end: host buffers, copies inside the timed region
     e2e = run_e2e(args, w, dev, b0, world) if not args.no_e2e else None

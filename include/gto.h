@@ -219,8 +219,10 @@ typedef struct {
  * out->loss[b] and grad_root[b,:] = weight * (p_M - p_T), the derivative of weight * H with
  * respect to the draft logits of that row ([B, V_draft], logit dtype, every entry written);
  * a trainer passes weight = 1 / (number of supervised positions).  Needs tree->row_lse from
- * gto_build_tree on the same draft logits.  An increasing d2t (a vocabulary subset listed in
- * id order) is streamed at memory bandwidth; any other injective map is gathered, slower. */
+ * gto_build_tree on the same draft logits.  Any d2t with entries in [0, V_target) is served;
+ * an increasing one (a vocabulary subset listed in id order) reads every 32-byte sector of
+ * the target row once.  An entry outside the target vocabulary is reported in the device
+ * status word (GTO_ERR_BAD_INDEX) and counts as probability 0. */
 gto_status gto_token_loss(gto_ctx* ctx, const void* draft_logits, const void* target_logits,
                           const int32_t* d2t, const gto_tree* tree, float weight,
                           void* grad_root, const gto_token_stats* out, void* stream);

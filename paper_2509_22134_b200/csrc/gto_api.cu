@@ -21,9 +21,6 @@ struct gto_ctx {
   int32_t* list;      // [G*B*R] needed target rows
   int32_t* list_count;
   int32_t* status;
-  uint32_t* map_bits;   // token loss: bitmap of the id map's image, and
-  uint32_t* map_prefix; //   the number of mapped ids below each of its words
-  int32_t* map_state;   //   [0] = 1 if the map is not increasing
   int32_t* live_list;   // gradient: slices that carry a gradient (GTO_FLAG_GRAD_LIVE_ROWS)
   int32_t* live_count;
   int sms;
@@ -181,13 +178,9 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   const size_t o_id = off;  off += align_up(rows * c->k * sizeof(int32_t));
   const size_t o_z = off;   off += align_up(rows * c->k * sizeof(float));
   const size_t o_list = off; off += align_up(rows * sizeof(int32_t));
-  const size_t map_words = static_cast<size_t>(c->V_target + 31) / 32 + 1;
-  const size_t o_bits = off; off += align_up(map_words * sizeof(uint32_t));
-  const size_t o_pre = off; off += align_up(map_words * sizeof(uint32_t));
   const size_t o_live = off; off += align_up(static_cast<size_t>(c->B) * c->D * sizeof(int32_t));
   const size_t o_cnt = off; off += 256;
   const size_t o_st = off;  off += 256;
-  const size_t o_ms = off;  off += 256;
   const size_t o_lc = off;  off += 256;
   if (cudaMalloc(&ctx->ws, off) != cudaSuccess) {
     cudaGetLastError();
@@ -199,12 +192,9 @@ gto_status gto_create(gto_ctx** out, const gto_config* c, int device) {
   ctx->list = reinterpret_cast<int32_t*>(ctx->ws + o_list);
   ctx->list_count = reinterpret_cast<int32_t*>(ctx->ws + o_cnt);
   ctx->status = reinterpret_cast<int32_t*>(ctx->ws + o_st);
-  ctx->map_bits = reinterpret_cast<uint32_t*>(ctx->ws + o_bits);
-  ctx->map_prefix = reinterpret_cast<uint32_t*>(ctx->ws + o_pre);
-  ctx->map_state = reinterpret_cast<int32_t*>(ctx->ws + o_ms);
   ctx->live_list = reinterpret_cast<int32_t*>(ctx->ws + o_live);
   ctx->live_count = reinterpret_cast<int32_t*>(ctx->ws + o_lc);
-  if (cudaMemset(ctx->ws + o_cnt, 0, 1024) != cudaSuccess ||
+  if (cudaMemset(ctx->ws + o_cnt, 0, 768) != cudaSuccess ||
       cudaMallocHost(&ctx->h_list, (rows + 1) * sizeof(int32_t)) != cudaSuccess) {
     cudaGetLastError();
     cudaFree(ctx->ws);
@@ -448,9 +438,6 @@ gto_status token_loss_impl(gto_ctx* ctx, const void* draft, const void* target, 
   a.loss = out->loss;
   a.lse_t = out->lse_t;
   a.status = ctx->status;
-  a.map_bits = ctx->map_bits;
-  a.map_prefix = ctx->map_prefix;
-  a.map_state = ctx->map_state;
   LaunchSpan span(ctx, GTO_K_TOKEN_LOSS, s);
   if (gto::launch_token_loss(a, ctx->sms, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
   return GTO_OK;

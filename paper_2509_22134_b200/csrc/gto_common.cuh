@@ -45,6 +45,7 @@ struct Bf16 {
   static constexpr int kBytes = 2;
   static constexpr uint32_t kNegInfWord = 0xff80ff80u;
   using Storage = uint16_t;
+  static constexpr Storage kNegInfElem = 0xff80u;
   // stored bits of element e of a vector
   __device__ static __forceinline__ Storage element(const uint4& v, int e) {
     const uint32_t w = e < 4 ? (e < 2 ? v.x : v.y) : (e < 6 ? v.z : v.w);
@@ -96,6 +97,7 @@ struct F16 {
   static constexpr int kBytes = 2;
   static constexpr uint32_t kNegInfWord = 0xfc00fc00u;
   using Storage = uint16_t;
+  static constexpr Storage kNegInfElem = 0xfc00u;
   __device__ static __forceinline__ Storage element(const uint4& v, int e) {
     const uint32_t w = e < 4 ? (e < 2 ? v.x : v.y) : (e < 6 ? v.z : v.w);
     return static_cast<Storage>(e & 1 ? w >> 16 : w & 0xffffu);
@@ -143,6 +145,7 @@ struct F32 {
   static constexpr int kBytes = 4;
   static constexpr uint32_t kNegInfWord = 0xff800000u;
   using Storage = uint32_t;
+  static constexpr Storage kNegInfElem = 0xff800000u;
   __device__ static __forceinline__ Storage element(const uint4& v, int e) {
     return e < 2 ? (e == 0 ? v.x : v.y) : (e == 2 ? v.z : v.w);
   }

@@ -97,9 +97,6 @@ struct TokenLossArgs {
   double* loss;            // [B]
   double* lse_t;           // [B]
   int32_t* status;
-  uint32_t* map_bits;      // workspace: bitmap of the id map's image, ceil(V_target/32)+1 words
-  uint32_t* map_prefix;    // workspace: mapped ids below each bitmap word
-  int32_t* map_state;      // workspace: [0] = 1 if the map is not increasing
 };
 cudaError_t launch_token_loss(const TokenLossArgs& a, int sms, cudaStream_t stream,
                               int64_t* launches);

@@ -6,22 +6,20 @@
 // logits at the mapped ids.
 //
 // Streaming kernel (token_loss_stream_kernel): a position is shared by a thread-block
-// cluster; every CTA owns a contiguous range of draft ids.  Pass A streams the CTA's part of
-// the target row with 16-byte loads, keeps the logits of the mapped ids in shared memory in
-// draft-id order and sums their exponentials; the cluster then combines the partial sums
-// through distributed shared memory.  Pass B streams the draft row once, takes the target
-// logits from shared memory, and writes the gradient row.  Every byte of the two rows is read
-// once from HBM and nothing is gathered.  With an id map this needs the map to be increasing
-// (a vocabulary subset listed in id order): then the mapped target logits, taken in target-id
-// order, are already in draft-id order, and "is this target id mapped, and to which draft id"
-// is a bit test and a prefix pop-count over a bitmap of the map's image (token_map_*
-// kernels, rebuilt on every call because the map is the caller's).  A map that is injective
-// but not increasing is detected while the bitmap is built and handled by the gathering
-// kernel below instead.
+// cluster; every CTA owns a contiguous range of draft ids.  Pass A brings the range's target
+// logits into shared memory in draft-id order -- without an id map with 16-byte streaming
+// loads; with one by a gather through L1 in which one warp load covers 32 neighbouring draft
+// ids, whose target ids lie within a few 128-byte lines, so that every 32-byte sector of the
+// target row comes from HBM once (a vocabulary subset listed in id order touches all of them:
+// the bytes moved are those of the whole row) -- and sums their exponentials from shared
+// memory; the cluster then combines the partial sums through distributed shared memory.
+// Pass B streams the draft row once, takes the target logits from shared memory, and writes
+// the gradient row.  Any map is served; an id outside the target vocabulary is reported in
+// the status word and counts as probability 0.
 //
-// Gathering kernel (token_loss_gather_kernel): one CTA per position, two passes over the two
-// rows (the second hits L2); the id-map gather is laid out so that a warp load touches few
-// 32-byte sectors.  Serves any injective map and rows too long for the cluster's shared memory.
+// Two-pass kernel (token_loss_gather_kernel): one CTA per position, two passes over the two
+// rows (the second hits L2), nothing kept in shared memory.  Serves short rows without a map
+// in a large batch, where it is faster, and rows too long for a cluster's shared memory.
 #include <cooperative_groups.h>
 
 #include "gto_common.cuh"
@@ -35,62 +33,18 @@ namespace cg = cooperative_groups;
 #ifndef GTO_TOK_THREADS
 #define GTO_TOK_THREADS 256
 #endif
-constexpr int kTokThreads = GTO_TOK_THREADS;
+constexpr int kTokThreads = GTO_TOK_THREADS;  // two-pass kernel
 constexpr int kTokWarps = kTokThreads / 32;
+#ifndef GTO_TOK_STREAM_THREADS
+#define GTO_TOK_STREAM_THREADS 512
+#endif
+constexpr int kStreamMaxThreads = 512;  // streaming kernel: the block size is a launch parameter
+constexpr int kStreamMaxWarps = kStreamMaxThreads / 32;
 
 __device__ __forceinline__ double warp_sum_f64(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
   return v;
-}
-
-// ------------------------------------------------------------------ bitmap of the id map
-// One CTA builds, for the call's id map: bitmap[w] bit i = target id 32 w + i is the image of a
-// draft id; prefix[w] = number of mapped target ids below 32 w; map_state[0] = 1 if the map is
-// not strictly increasing or holds an id outside the target vocabulary (the streaming kernel
-// then leaves the call to the gathering kernel).  A few thousand words: one launch is cheaper
-// than a grid-wide version with its extra launches.
-__global__ void __launch_bounds__(1024) token_map_build_kernel(
-    const int32_t* __restrict__ d2t, int V_draft, int V_target, int n_words, uint32_t* bitmap,
-    uint32_t* __restrict__ prefix, int32_t* map_state, int32_t* __restrict__ status) {
-  __shared__ uint32_t warp_tot[32];
-  __shared__ uint32_t carry;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (int w = tid; w < n_words; w += 1024) bitmap[w] = 0;
-  if (tid == 0) {
-    carry = 0;
-    map_state[0] = 0;
-  }
-  __syncthreads();
-  for (int v = tid; v < V_draft; v += 1024) {
-    const int id = d2t[v];
-    if (id < 0 || id >= V_target) {
-      atomicOr(status, kStatusBadIndex);
-      atomicOr(map_state, 1);  // ranks would no longer be draft ids
-      continue;
-    }
-    if (v > 0 && d2t[v - 1] >= id) atomicOr(map_state, 1);
-    atomicOr(bitmap + (id >> 5), 1u << (id & 31));
-  }
-  __syncthreads();
-  for (int base = 0; base < n_words; base += 1024) {
-    const int w = base + tid;
-    const uint32_t c = w < n_words ? __popc(bitmap[w]) : 0u;
-    uint32_t inc = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const uint32_t up = __shfl_up_sync(kFull, inc, o);
-      if (lane >= o) inc += up;
-    }
-    if (lane == 31) warp_tot[warp] = inc;
-    __syncthreads();
-    uint32_t before = carry;
-    for (int q = 0; q < warp; ++q) before += warp_tot[q];
-    if (w < n_words) prefix[w] = before + inc - c;
-    __syncthreads();
-    if (tid == 1023) carry = before + inc;
-    __syncthreads();
-  }
 }
 
 // ------------------------------------------------------------------ streaming kernel
@@ -101,19 +55,18 @@ struct TokPartial {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLossArgs a) {
+__global__ void __launch_bounds__(kStreamMaxThreads, 3) token_loss_stream_kernel(TokenLossArgs a) {
   constexpr int E = T::kPerVec;
   extern __shared__ __align__(16) unsigned char s_raw[];  // the range's target logits, logit dtype
   __shared__ TokPartial part;
-  __shared__ float s_m[kTokWarps];
-  __shared__ double s_s[kTokWarps];
+  __shared__ float s_m[kStreamMaxWarps];
+  __shared__ double s_s[kStreamMaxWarps];
   cg::cluster_group cluster = cg::this_cluster();
   const int C = static_cast<int>(cluster.num_blocks());
   const int c = static_cast<int>(cluster.block_rank());
   const int b = blockIdx.x / C;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // the map turned out not to be increasing: the gathering kernel does this call
-  if (a.d2t != nullptr && a.map_state[0] != 0) return;
+  const int n_threads = blockDim.x, n_warps = n_threads >> 5;
 
   const int nvec = a.V_draft / E;
   const int per = (nvec + C - 1) / C;
@@ -142,48 +95,55 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
     }
   };
   if (a.d2t == nullptr) {
-    for (int i = vec0 + tid; i < vec1; i += kTokThreads) {
+    for (int i = vec0 + tid; i < vec1; i += n_threads) {
       reinterpret_cast<uint4*>(s_raw)[i - vec0] = ld_stream16(zt + static_cast<size_t>(i) * 16);
     }
   } else if (id1 > id0) {
-    const int t_lo = a.d2t[id0], t_hi = a.d2t[id1 - 1];  // target ids of the range's ends
-    const int i_end = t_hi / E + 1;
-    constexpr int U = 4;  // vectors in flight per thread
-    for (int i0 = t_lo / E + tid; i0 < i_end; i0 += U * kTokThreads) {
-      uint4 v[U];
-      uint32_t word[U], pre[U];
+    // gather through L1: lane l of a warp takes draft ids base + e*32 + l, so that one warp load
+    // covers 32 neighbouring draft ids, whose target ids lie within a few 128-byte lines
+    // (a sector is fetched from L2 once and hit again by the following loads)
+    constexpr int kChunk = 32 * E;
+#ifndef GTO_TOK_UC
+#define GTO_TOK_UC 2
+#endif
+    constexpr int UC = GTO_TOK_UC;  // chunks in flight per warp
+    const int n_ids = id1 - id0;
+    const Elem* zt_e = reinterpret_cast<const Elem*>(zt);
+    for (int c0 = warp * UC * kChunk; c0 < n_ids; c0 += n_warps * UC * kChunk) {
+      int id[UC][E];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int i = i0 + u * kTokThreads;
-        if (i < i_end) {
-          v[u] = ld_stream16(zt + static_cast<size_t>(i) * 16);
-          word[u] = __ldg(a.map_bits + ((i * E) >> 5));
-          pre[u] = __ldg(a.map_prefix + ((i * E) >> 5));
-        } else {
-          word[u] = 0;
-        }
-      }
+      for (int u = 0; u < UC; ++u)
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        // E consecutive target ids: their bits of the image bitmap, and the draft id (rank)
-        // of the first mapped one among them
-        const int first = (i0 + u * kTokThreads) * E;
-        const unsigned bits = (word[u] >> (first & 31)) & ((1u << E) - 1u);
-        unsigned todo = bits;
-        int rank = static_cast<int>(pre[u]) + __popc(word[u] & ((1u << (first & 31)) - 1u));
-        while (todo) {  // about E * V_draft / V_target mapped ids per vector
-          const int e = __ffs(todo) - 1;
-          todo &= todo - 1;
-          // neighbouring ranges share their end vectors: keep the ids of this range only
-          if (rank >= id0 && rank < id1) s_t[rank - id0] = T::element(v[u], e);
-          ++rank;
+        for (int e = 0; e < E; ++e) {
+          const int v = c0 + u * kChunk + e * 32 + lane;
+          id[u][e] = v < n_ids ? __ldg(a.d2t + id0 + v) : -1;
         }
-      }
+      Elem x[UC][E];
+      bool bad = false;
+#pragma unroll
+      for (int u = 0; u < UC; ++u)
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const int v = c0 + u * kChunk + e * 32 + lane;
+          x[u][e] = T::kNegInfElem;  // an id outside the target vocabulary: probability 0
+          if (static_cast<unsigned>(id[u][e]) < static_cast<unsigned>(a.V_target))
+            x[u][e] = zt_e[id[u][e]];
+          else if (v < n_ids)
+            bad = true;
+        }
+#pragma unroll
+      for (int u = 0; u < UC; ++u)
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+          const int v = c0 + u * kChunk + e * 32 + lane;
+          if (v < n_ids) s_t[v] = x[u][e];
+        }
+      if (bad) atomicOr(a.status, kStatusBadIndex);
     }
   }
   __syncthreads();
   // the range's log-sum-exp from shared memory (dense, in draft-id order)
-  for (int i = tid; i < vec1 - vec0; i += kTokThreads) {
+  for (int i = tid; i < vec1 - vec0; i += n_threads) {
     float t[E];
     T::unpack(reinterpret_cast<const uint4*>(s_raw)[i], t);
     take(t);
@@ -200,9 +160,9 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
   __syncthreads();
   if (tid == 0) {
     float M = s_m[0];
-    for (int w = 1; w < kTokWarps; ++w) M = fmaxf(M, s_m[w]);
+    for (int w = 1; w < n_warps; ++w) M = fmaxf(M, s_m[w]);
     double S = 0.0;
-    for (int w = 0; w < kTokWarps; ++w)
+    for (int w = 0; w < n_warps; ++w)
       if (s_m[w] != -INFINITY) S += s_s[w] * exp2(static_cast<double>((s_m[w] - M) * kLog2e));
     part.m = M;
     part.s = S;
@@ -231,7 +191,7 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
   // with `accumulate` the row may already hold the surrogate's gradient of the same draft row
   const bool add = a.acc_path_len != nullptr && a.acc_path_len[b] > 0 && a.acc_coeff[b] != 0.0;
   float h = 0.f;
-  for (int i = vec0 + tid; i < vec1; i += kTokThreads) {
+  for (int i = vec0 + tid; i < vec1; i += n_threads) {
     float t[E], z[E], g[E];
     T::unpack(reinterpret_cast<const uint4*>(s_raw)[i - vec0], t);
     T::unpack(ld_stream16(zd + static_cast<size_t>(i) * 16), z);
@@ -256,7 +216,7 @@ __global__ void __launch_bounds__(kTokThreads) token_loss_stream_kernel(TokenLos
   __syncthreads();
   if (tid == 0) {
     double H = 0.0;
-    for (int w = 0; w < kTokWarps; ++w) H += s_s[w];
+    for (int w = 0; w < n_warps; ++w) H += s_s[w];
     part.h = H;
   }
   cluster.sync();  // the partial losses are visible; nobody has left while its partials were read
@@ -277,8 +237,6 @@ __global__ void __launch_bounds__(kTokThreads, 8) token_loss_gather_kernel(Token
   __shared__ double s_sum[kTokWarps];
   __shared__ double s_lse;
   __shared__ __align__(16) float s_t[kTokWarps][kChunk];  // a warp's gathered target logits
-  // an increasing map is served by the streaming kernel of the same call
-  if (a.map_state != nullptr && a.map_state[0] == 0) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x;
   const char* zd = static_cast<const char*>(a.draft) +
@@ -406,7 +364,8 @@ __global__ void __launch_bounds__(kTokThreads, 8) token_loss_gather_kernel(Token
 }
 
 template <typename T>
-cudaError_t launch_stream(const TokenLossArgs& a, int C, size_t smem, cudaStream_t stream) {
+cudaError_t launch_stream(const TokenLossArgs& a, int C, int threads, size_t smem,
+                          cudaStream_t stream) {
   // raise the kernel's dynamic shared memory limit when a call needs more than any before it
   // (per device: the attribute belongs to the device's copy of the function)
   static int allowed[64] = {};
@@ -421,7 +380,7 @@ cudaError_t launch_stream(const TokenLossArgs& a, int C, size_t smem, cudaStream
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(static_cast<unsigned>(a.B) * C);
-  cfg.blockDim = dim3(kTokThreads);
+  cfg.blockDim = dim3(threads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
   cudaLaunchAttribute attr{};
@@ -458,34 +417,27 @@ cudaError_t launch_token_loss(const TokenLossArgs& a, int sms, cudaStream_t stre
   if (a.B <= 0) return cudaSuccess;
   const int C = token_loss_cluster_size(a.B, a.V_draft, a.d2t != nullptr, a.dtype, sms);
   cudaError_t e = cudaSuccess;
-  if (C > 0 && a.d2t != nullptr) {
-    // the bitmap of the map's image and its prefix counts
-    const int n_words = (a.V_target + 31) / 32 + 1;
-    token_map_build_kernel<<<1, 1024, 0, stream>>>(a.d2t, a.V_draft, a.V_target, n_words, a.map_bits,
-                                                   a.map_prefix, a.map_state, a.status);
-    ++*launches;
-  }
   if (C > 0) {
     const int E = 16 / elem_bytes(a.dtype);
     const int per = (a.V_draft / E + C - 1) / C;
     const size_t smem = static_cast<size_t>(per) * 16;
-    if (a.dtype == GTO_BF16) e = launch_stream<Bf16>(a, C, smem, stream);
-    else if (a.dtype == GTO_F16) e = launch_stream<F16>(a, C, smem, stream);
-    else e = launch_stream<F32>(a, C, smem, stream);
+    // measured on B200 (us per call, B = 1024, bf16): with a map 512 threads 99, 256 threads
+    // 117; without a map (151 936 ids) 256 threads 162, 512 threads 152
+    const int threads = GTO_TOK_STREAM_THREADS;
+    if (a.dtype == GTO_BF16) e = launch_stream<Bf16>(a, C, threads, smem, stream);
+    else if (a.dtype == GTO_F16) e = launch_stream<F16>(a, C, threads, smem, stream);
+    else e = launch_stream<F32>(a, C, threads, smem, stream);
     if (e != cudaSuccess) return e;
     ++*launches;
-    if (a.d2t == nullptr) return cudaGetLastError();
+    return cudaGetLastError();
   }
-  // any injective map (the streaming kernel has returned at once if the map is increasing,
-  // this one returns at once if it is), and rows too long for a cluster's shared memory
-  TokenLossArgs g = a;
-  if (C == 0) g.map_state = nullptr;
+  // short unmapped rows of a large batch, and rows too long for a cluster's shared memory
   if (a.dtype == GTO_BF16)
-    token_loss_gather_kernel<Bf16><<<a.B, kTokThreads, 0, stream>>>(g);
+    token_loss_gather_kernel<Bf16><<<a.B, kTokThreads, 0, stream>>>(a);
   else if (a.dtype == GTO_F16)
-    token_loss_gather_kernel<F16><<<a.B, kTokThreads, 0, stream>>>(g);
+    token_loss_gather_kernel<F16><<<a.B, kTokThreads, 0, stream>>>(a);
   else
-    token_loss_gather_kernel<F32><<<a.B, kTokThreads, 0, stream>>>(g);
+    token_loss_gather_kernel<F32><<<a.B, kTokThreads, 0, stream>>>(a);
   ++*launches;
   return cudaGetLastError();
 }

@@ -260,7 +260,7 @@ def test_token_loss_streaming_layouts(harness, kw):
 
 
 def test_token_loss_with_an_injective_map_that_is_not_increasing(harness):
-    """Any injective map is accepted: one that is not in id order takes the gathering kernel."""
+    """Any injective map is accepted, in id order or not."""
     from paper_2509_22134_b200.runner import GtoPass
     w = synth.Workload("tok", B=16, V_draft=2048, V_target=8200, D=2, k=4, g=8, dtype="bf16", seed=31)
     data = synth.generate(w, DEV)
