@@ -35,9 +35,6 @@ namespace cg = cooperative_groups;
 #endif
 constexpr int kTokThreads = GTO_TOK_THREADS;  // two-pass kernel
 constexpr int kTokWarps = kTokThreads / 32;
-#ifndef GTO_TOK_PF
-#define GTO_TOK_PF 1  // bulk L2 prefetch of a CTA's share of the rows at its start
-#endif
 #ifndef GTO_TOK_STREAM_THREADS
 #define GTO_TOK_STREAM_THREADS 512
 #endif
@@ -82,38 +79,6 @@ __global__ void __launch_bounds__(kStreamMaxThreads, 3) token_loss_stream_kernel
   using Elem = typename T::Storage;
   Elem* s_t = reinterpret_cast<Elem*>(s_raw);
 
-#if GTO_TOK_PF
-  // Ask for the CTA's part of the two rows to be brought into L2 now (one instruction per 16 KB,
-  // no registers or shared memory hold the data): the loads below then find most of it there
-  // instead of each paying a DRAM access, and pass B's draft loads, which otherwise start only
-  // after the cluster's barrier, find all of it.
-  {
-    constexpr int kPfBytes = 16384;
-    auto prefetch = [&](const char* base, long long bytes) {
-      for (long long off = static_cast<long long>(tid) * kPfBytes; off < bytes;
-           off += static_cast<long long>(n_threads) * kPfBytes) {
-        const long long rest = bytes - off;
-        const int n = static_cast<int>(rest < kPfBytes ? rest : kPfBytes) & ~15;
-        if (n > 0)
-          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(base + off), "r"(n)
-                       : "memory");
-      }
-    };
-    if (a.d2t == nullptr) {
-      prefetch(zt + static_cast<size_t>(vec0) * 16, static_cast<long long>(vec1 - vec0) * 16);
-    } else if (id1 > id0) {
-      const int t_lo = a.d2t[id0], t_hi = a.d2t[id1 - 1];
-      // an id map in id order: the range's target ids are one stretch of the row
-      if (t_lo >= 0 && t_hi < a.V_target && t_hi >= t_lo &&
-          static_cast<long long>(t_hi - t_lo) <= 2ll * (id1 - id0) * (a.V_target / a.V_draft + 1)) {
-        const long long lo = (static_cast<long long>(t_lo) * T::kBytes) & ~15ll;
-        const long long hi = (static_cast<long long>(t_hi + 1) * T::kBytes) & ~15ll;
-        prefetch(zt + lo, hi - lo);
-      }
-    }
-    prefetch(zd + static_cast<size_t>(vec0) * 16, static_cast<long long>(vec1 - vec0) * 16);
-  }
-#endif
   // ---- pass A: the range's mapped target logits into shared memory, then their max and sum
   float m = -INFINITY, s = 0.f;
   auto take = [&](const float (&t)[E]) {
@@ -456,9 +421,10 @@ cudaError_t launch_token_loss(const TokenLossArgs& a, int sms, cudaStream_t stre
     const int E = 16 / elem_bytes(a.dtype);
     const int per = (a.V_draft / E + C - 1) / C;
     const size_t smem = static_cast<size_t>(per) * 16;
-    // measured on B200 (us per call, B = 1024, bf16): with a map 512 threads 99, 256 threads
-    // 117; without a map (151 936 ids) 256 threads 162, 512 threads 152
-    const int threads = GTO_TOK_STREAM_THREADS;
+    // measured on B200 (us per call, bf16): B = 1024 with a map 512 threads 99, 256 threads
+    // 117; without a map (151 936 ids) 512 threads 152, 256 threads 162; B = 64 with a map
+    // 512 threads 27, 256 threads 16
+    const int threads = a.B >= 2 * sms ? GTO_TOK_STREAM_THREADS : 256;
     if (a.dtype == GTO_BF16) e = launch_stream<Bf16>(a, C, threads, smem, stream);
     else if (a.dtype == GTO_F16) e = launch_stream<F16>(a, C, threads, smem, stream);
     else e = launch_stream<F32>(a, C, threads, smem, stream);

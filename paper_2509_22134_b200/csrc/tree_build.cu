@@ -48,6 +48,8 @@ struct TreeSmem {
   int fpool[kMaxDepth][kMaxTopK];       // fpool[d][j]: pool index of frontier slot j at depth d
   unsigned selmask[kMaxDepth][kMaskWords];  // selected candidates of each layer, bit q
   int sel_before[kMaxDepth + 1];        // selected nodes in the layers before this one
+  int sel_base[kMaxDepth];              // selected candidates of a layer known after the probes
+  int sel_count[kMaxDepth];             // selected candidates of a layer
   int parent[kMaxNodes];
 };
 
@@ -166,23 +168,12 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
     cur ^= 1;
   }
 
-  // ---- global top-g: rank among all candidates = rank in the layer + entries ahead in
-  //      every other layer.  Items are (layer l, rank r < min(len, g)), dealt round-robin.
-  int n_items = 0;
-  for (int l = 0; l < D; ++l) n_items += min(list_len(l), g);
-  auto item = [&](int t, int& l, int& r) {
-    l = 0;
-    int n = min(list_len(0), g);
-    while (t >= n) {
-      t -= n;
-      ++l;
-      n = min(list_len(l), g);
-    }
-    r = t;
-  };
-  for (int t = tid; t < n_items; t += kTreeThreads) {
-    int l, r;
-    item(t, l, r);
+  // ---- global top-g.  A candidate's rank among all candidates = its rank in its layer +
+  //      the entries ahead of it in every other layer, and it grows with the layer rank, so the
+  //      selected candidates of a layer are its first s_l.  s_l is found in two rounds instead
+  //      of ranking every candidate that could be selected: kProbes evenly spaced layer ranks
+  //      bracket it, then the ranks inside the bracket are evaluated.
+  auto global_rank = [&](int l, int r) {
     const uint64_t x = skey[list_off(l) + r];
     int rank = r;
     if constexpr (K > 0) {
@@ -193,29 +184,66 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
       for (int lp = 0; lp < D && rank < g; ++lp)
         if (lp != l) rank += count_ahead(skey + list_off(lp), list_len(lp), x, lp < l);
     }
-    if (rank < g) {
-      const int q = sq[list_off(l) + r];
-      atomicOr(&sm.selmask[l][q >> 5], 1u << (q & 31));
+    return rank;
+  };
+  constexpr int kProbes = 8;
+  static_assert(kMaxDepth * kProbes <= kTreeThreads, "one thread per probe");
+  const int cap0 = min(k, g), cap1 = min(kk, g);  // candidates of a layer that can be selected
+  const int step0 = (cap0 + kProbes - 1) / kProbes, step1 = (cap1 + kProbes - 1) / kProbes;
+  {
+    // round 1: probe j of layer l looks at layer rank (j + 1) * step - 1
+    const int l = tid / kProbes, j = tid % kProbes;
+    bool sel = false;
+    if (l < D) {
+      const int r = (j + 1) * (l == 0 ? step0 : step1) - 1;
+      if (r < (l == 0 ? cap0 : cap1)) sel = global_rank(l, r) < g;
+    }
+    // the probes of a layer are kProbes neighbouring lanes; the selected ones come first
+    const unsigned mine = (__ballot_sync(kFull, sel) >> ((tid & 31) & ~(kProbes - 1))) &
+                          ((1u << kProbes) - 1u);
+    if (l < D && j == 0) {
+      const int base = __popc(mine) * (l == 0 ? step0 : step1);
+      sm.sel_base[l] = base;
+      sm.sel_count[l] = base;
     }
   }
   __syncthreads();
-  if (tid <= D) {
+  {
+    // round 2: the layer ranks from the last selected probe up to the next probe
+    const int n_items = step0 + (D - 1) * step1;
+    for (int t = tid; t < n_items; t += kTreeThreads) {
+      const int l = t < step0 ? 0 : 1 + (t - step0) / step1;
+      const int i = t < step0 ? t : (t - step0) % step1;
+      const int r = sm.sel_base[l] + i;
+      if (r < (l == 0 ? cap0 : cap1) && global_rank(l, r) < g) atomicAdd(&sm.sel_count[l], 1);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
     int n = 0;
-    for (int l = 0; l < tid; ++l)
-#pragma unroll
-      for (int w = 0; w < kMaskWords; ++w) n += __popc(sm.selmask[l][w]);
-    sm.sel_before[tid] = n;
+    for (int l = 0; l < D; ++l) {
+      sm.sel_before[l] = n;
+      n += sm.sel_count[l];
+    }
+    sm.sel_before[D] = n;  // = g
+  }
+  __syncthreads();
+  // one thread per selected candidate: (layer l, layer rank r)
+  const int n_sel = sm.sel_before[D];
+  int l = 0, r = 0, q = 0;
+  const bool mine = tid < n_sel;
+  if (mine) {
+    while (tid >= sm.sel_before[l + 1]) ++l;
+    r = tid - sm.sel_before[l];
+    q = sq[list_off(l) + r];
+    atomicOr(&sm.selmask[l][q >> 5], 1u << (q & 31));
   }
   __syncthreads();
 
   // ---- per-node fields, listed in ascending pool index
   const size_t obase = static_cast<size_t>(tree) * g;
-  for (int t = tid; t < n_items; t += kTreeThreads) {
-    int l, r;
-    item(t, l, r);
+  if (mine) {
     const int off = list_off(l);
-    const int q = sq[off + r];
-    if (!((sm.selmask[l][q >> 5] >> (q & 31)) & 1u)) continue;
     const int n = sm.sel_before[l] + bits_below(sm.selmask[l], q);
     const int depth = l + 1;
     int c = q, ctx = 0, par = -1;
