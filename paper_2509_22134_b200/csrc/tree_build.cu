@@ -12,7 +12,7 @@
 // number of entries ahead of it (a binary search again); only the first g of a layer can
 // reach the global top-g.  Ties go to the lower index everywhere: child index within a
 // parent, parent slot within a layer, layer (= depth) across layers, i.e. the pool index.
-// Scores are fp64 sums of min(z - lse, 0), so a ranking differs from an exact evaluation only
+// Scores are fp64 sums of min(z - lse, 0), compared as fp64, so a ranking differs from an exact evaluation only
 // where two scores agree to ~1e-7.  The clamp matters: a log-probability is never positive,
 // but the fp32-accumulated log-sum-exp of a row with one dominant logit can come out a few
 // 1e-7 below that logit; without the clamp such a child would outscore its own parent and
@@ -33,17 +33,15 @@ __device__ __forceinline__ double edge_logp(float z, double lse) {
   return fmin(static_cast<double>(z) - lse, 0.0);
 }
 
-__device__ __forceinline__ uint64_t score_key(double s) {
-  uint64_t u = static_cast<uint64_t>(__double_as_longlong(s + 0.0));
-  return u ^ ((u >> 63) ? ~0ull : (1ull << 63));
-}
-__device__ __forceinline__ double key_score(uint64_t k) {
-  uint64_t u = k ^ ((k >> 63) ? (1ull << 63) : ~0ull);
-  return __longlong_as_double(static_cast<long long>(u));
+// The next double above x (x is a score: finite or -inf, never -0 or NaN in a valid tree), so
+// that "y > x" can be asked as "y >= next_above(x)".
+__device__ __forceinline__ double next_above(double x) {
+  const long long b = __double_as_longlong(x);
+  return __longlong_as_double(b < 0 ? b - 1 : b + 1);
 }
 
 struct TreeSmem {
-  uint64_t ukey[kMaxLayer];             // keys of the layer in work, by candidate index q
+  double uscore[kMaxLayer];             // scores of the layer in work, by candidate index q
   double fcum[2][kMaxTopK];             // cumulative score of the frontier (double-buffered)
   int fpool[kMaxDepth][kMaxTopK];       // fpool[d][j]: pool index of frontier slot j at depth d
   unsigned selmask[kMaxDepth][kMaskWords];  // selected candidates of each layer, bit q
@@ -53,11 +51,11 @@ struct TreeSmem {
   int parent[kMaxNodes];
 };
 
-// Entries of a descending list that come before x; equal keys come before x iff `ties_first`.
-__device__ __forceinline__ int count_ahead(const uint64_t* list, int n, uint64_t x,
-                                           bool ties_first) {
-  // x + 1 turns "y >= x" into "y > x": keys of finite scores never reach ~0
-  const uint64_t bound = ties_first ? x : x + 1;  // ahead iff y >= bound
+// Entries of a descending list that come before x; equal scores come before x iff `ties_first`.
+// The comparisons are fp64 compares (the fp64 pipe is otherwise idle in this kernel, while a
+// 64-bit integer compare costs two instructions on the ALU pipe, which bounds it).
+__device__ __forceinline__ int count_ahead(const double* list, int n, double x, bool ties_first) {
+  const double bound = ties_first ? x : next_above(x);  // ahead iff y >= bound
   int lo = 0, hi = n;
   while (lo < hi) {
     const int mid = (lo + hi) >> 1;
@@ -69,9 +67,8 @@ __device__ __forceinline__ int count_ahead(const uint64_t* list, int n, uint64_t
 // Same for a list of compile-time length N: a fixed number of branch-free steps (the answer
 // is built bit by bit from the top).
 template <int N>
-__device__ __forceinline__ int count_ahead_fixed(const uint64_t* list, uint64_t x,
-                                                 bool ties_first) {
-  const uint64_t bound = ties_first ? x : x + 1;
+__device__ __forceinline__ int count_ahead_fixed(const double* list, double x, bool ties_first) {
+  const double bound = ties_first ? x : next_above(x);
   constexpr int kTopBit = N >= 128 ? 128 : N >= 64 ? 64 : N >= 32 ? 32 : N >= 16 ? 16
                           : N >= 8 ? 8 : N >= 4 ? 4 : N >= 2 ? 2 : 1;
   static_assert(N < 256, "step table");
@@ -104,8 +101,8 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
   const int tree = blockIdx.x;
   const int D = a.D, k = K > 0 ? K : a.k, g = a.g, R = a.R, kk = k * k;
   const int P = k + (D - 1) * kk;
-  uint64_t* skey = reinterpret_cast<uint64_t*>(dyn);       // [P] every layer, sorted
-  double* lse = reinterpret_cast<double*>(skey + P);        // [R] staged row log-sum-exps
+  double* skey = reinterpret_cast<double*>(dyn);           // [P] scores of every layer, sorted
+  double* lse = skey + P;                                   // [R] staged row log-sum-exps
   float* top_z = reinterpret_cast<float*>(lse + R);        // [R*k] staged top-k logits
   uint8_t* sq = reinterpret_cast<uint8_t*>(top_z + R * k); // [P] candidate index at that rank
   const int32_t* top_id = a.top_id + static_cast<size_t>(tree) * R * k;
@@ -123,8 +120,8 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
   __syncthreads();
   // ---- depth 1: the root's k best tokens, already in rank order = pool order
   if (tid < k) {
-    const double sc = edge_logp(top_z[tid], lse[0]);
-    skey[tid] = score_key(sc);
+    const double sc = edge_logp(top_z[tid], lse[0]) + 0.0;  // -0 -> +0
+    skey[tid] = sc;
     sq[tid] = static_cast<uint8_t>(tid);
     if (D > 1) {
       sm.fcum[0][tid] = sc;
@@ -139,12 +136,10 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
     const int base = list_off(d - 1);
     const int j = tid / k, c = tid - j * k;
     double sc = 0.0;
-    uint64_t key = 0;
     if (tid < kk) {
       const int row = 1 + (d - 2) * k + j;
-      sc = sm.fcum[cur][j] + edge_logp(top_z[row * k + c], lse[row]);
-      key = score_key(sc);
-      sm.ukey[tid] = key;
+      sc = sm.fcum[cur][j] + edge_logp(top_z[row * k + c], lse[row]) + 0.0;
+      sm.uscore[tid] = sc;
     }
     __syncthreads();
     if (tid < kk) {
@@ -152,12 +147,12 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
       if constexpr (K > 0) {
 #pragma unroll
         for (int jp = 0; jp < K; ++jp)
-          if (jp != j) rank += count_ahead_fixed<K>(&sm.ukey[jp * K], key, jp < j);
+          if (jp != j) rank += count_ahead_fixed<K>(&sm.uscore[jp * K], sc, jp < j);
       } else {
         for (int jp = 0; jp < k; ++jp)
-          if (jp != j) rank += count_ahead(&sm.ukey[jp * k], k, key, jp < j);
+          if (jp != j) rank += count_ahead(&sm.uscore[jp * k], k, sc, jp < j);
       }
-      skey[base + rank] = key;
+      skey[base + rank] = sc;
       sq[base + rank] = static_cast<uint8_t>(tid);
       if (d < D && rank < k) {
         sm.fcum[cur ^ 1][rank] = sc;
@@ -174,7 +169,7 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
   //      of ranking every candidate that could be selected: kProbes evenly spaced layer ranks
   //      bracket it, then the ranks inside the bracket are evaluated.
   auto global_rank = [&](int l, int r) {
-    const uint64_t x = skey[list_off(l) + r];
+    const double x = skey[list_off(l) + r];
     int rank = r;
     if constexpr (K > 0) {
       if (l != 0) rank += count_ahead_fixed<K>(skey, x, true);
@@ -263,7 +258,7 @@ __global__ void __launch_bounds__(kTreeThreads, 16) tree_build_kernel(TreeBuildA
     a.out.node_slot[obase + n] = (depth < D && r < k) ? r : -1;  // frontier slot = layer rank
     a.out.node_pool[obase + n] = off + q;
     a.out.node_logp[obase + n] = static_cast<float>(edge_logp(top_z[ctx * k + c], lse[ctx]));
-    a.out.node_score[obase + n] = key_score(skey[off + r]);
+    a.out.node_score[obase + n] = skey[off + r];
   }
   __syncthreads();
 
