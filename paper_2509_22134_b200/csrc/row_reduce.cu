@@ -15,14 +15,21 @@
 //
 // Selection without sorting: while streaming, each thread keeps only the largest and the
 // second largest of its batch maxima (a batch = kUnroll vectors loaded together) and which
-// batch held the largest.  From every warp's ceil(k / warps) largest thread maxima
-// the k-th largest is a lower bound tau of the row's k-th largest value (they are distinct
-// elements), so the row's top-k are among the elements >= tau, and only threads whose
-// maximum reaches tau can hold any.  Such a thread reloads its best batch (L2 hits, one
-// round trip) and pushes (value, id) candidates; if its second-best batch reaches tau too,
-// its warp rescans all of the thread's vectors cooperatively instead.  Each candidate's
-// rank among the candidates is then counted directly.  A row with more candidates than the
-// buffer holds (massive ties) takes k exact arg-max rounds.
+// batch held the largest, and leaves them in shared memory at the end of the row.  One warp
+// then selects: the k-th largest of the thread maxima is a lower bound tau of the row's k-th
+// largest value (they are k distinct elements), so the row's top-k are among the elements
+// >= tau, and only threads whose maximum reaches tau can hold any.  The best batch of such a
+// thread is fetched again, a lane per 16-byte vector, so all of them share one round trip;
+// if the thread's second-best batch reaches tau too, its whole share of the row is scanned
+// instead.  Every element >= tau becomes a (value, id) candidate, and a candidate's rank among
+// the candidates is counted directly.  A row with more candidates than the buffer holds
+// (massive ties) takes k exact arg-max rounds.  Selecting on one warp instead of letting every
+// warp handle its own threads costs a quarter of the instructions (the work is a dozen
+// elements, but a warp pays for its divergent lanes); the log-sum-exp is finished meanwhile
+// by a lane of another warp.  What the selection still costs is mostly the fetch: measured
+// on B200 at 64 KB rows, the pass without any selection runs 8 % faster, of which 6 % are the
+// re-fetched 32-byte sectors and the ranking, 1.6 % the hand-over and tau, 0.7 % the
+// log-sum-exp epilogue.
 //
 // Few rows (a small batch): one CTA per row leaves most SMs idle and a CTA alone is bound
 // by its own load latency, so the row is split over a thread-block cluster of kSplit CTAs,
@@ -53,13 +60,11 @@ namespace cg = cooperative_groups;
 #endif
 constexpr int kThreads = GTO_ROW_THREADS;
 constexpr int kWarps = kThreads / kWarp;
-constexpr int kMaxPer = (kMaxTopK + kWarps - 1) / kWarps;  // thread maxima kept per warp
 constexpr int kUnroll = GTO_ROW_UNROLL;
 constexpr int kMinCtas = GTO_ROW_MIN_CTAS;  // resident CTAs per SM the register budget allows
-constexpr int kCandCap = 1024;
+constexpr int kCandCap = 512;  // with the rest of RowSmem: 12 CTAs stay within 132 KB per SM
 constexpr float kRebase = 8.f;  // largest exponent argument before a thread moves its reference
 
-static_assert(kMaxPer * kWarps <= 32, "one lane per kept maximum");
 constexpr uint32_t kKeyNegInf = 0x007fffffu;  // orderable(-inf): stands for "no element"
 
 constexpr int kSplit = 4;  // CTAs (one cluster) per row in the split variant
@@ -73,11 +78,13 @@ struct RowPartial {
 };
 
 struct RowSmem {
-  uint32_t warp_top[kMaxPer * kWarps];  // each warp's largest thread maxima, as orderable keys
+  float tb1[kThreads];  // per thread: largest batch maximum,
+  float tb2[kThreads];  //   second largest,
+  int ti1[kThreads];    //   batch that held the largest
   float warp_sum[kWarps];
   float warp_ref[kWarps];
-  float tau;  // lower bound of the row's k-th largest value
   int n_cand;
+  unsigned short work[kThreads];  // threads whose best batch is fetched again
   unsigned long long cand[kCandCap];  // (value, id) keys
   unsigned long long round_best[kWarps];
   unsigned long long prev_key;
@@ -213,17 +220,12 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
     add_terms(v);
   }
 
-  // ---- warp level: the warp's `per` largest thread maxima, partial sum
-  const int per = (k + kWarps - 1) / kWarps;  // per * kWarps >= k distinct elements
+  // ---- hand-over: every thread's best and second-best batch maximum and best batch, and the
+  //      warp's partial sum (thread sums shifted to the warp's largest reference)
+  sm.tb1[tid] = b1;
+  sm.tb2[tid] = b2;
+  sm.ti1[tid] = i1;
   {
-    uint32_t key = orderable(b1);
-    for (int p = 0; p < per; ++p) {
-      const uint32_t top = __reduce_max_sync(kFull, key);
-      if (lane == 0) sm.warp_top[warp * kMaxPer + p] = top;
-      const unsigned holders = __ballot_sync(kFull, key == top);
-      if (lane == __ffs(holders) - 1) key = kKeyNegInf;
-    }
-    // shift the thread sums to the warp's largest reference, then add them
     const float wref = from_orderable(__reduce_max_sync(kFull, orderable(ref)));
     const float part = warp_sum_f32(s * ex2_approx(ref - wref));
     if (lane == 0) {
@@ -233,41 +235,101 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
   }
   __syncthreads();
 
-  // ---- warp 0: tau = the k-th largest of the warps' top maxima (each lane counts the
-  //      entries that precede its own in (value desc, lane asc) order)
-  if (warp == 0) {
-    const int n = per * kWarps;
-    uint32_t key = kKeyNegInf;
-    if (lane < n) key = sm.warp_top[(lane / per) * kMaxPer + lane % per];
-    int rank = 0;
-    for (int j = 0; j < n; ++j) {
-      const uint32_t o = __shfl_sync(kFull, key, j);
-      rank += (o > key || (o == key && j < lane)) ? 1 : 0;
+  // ---- row log-sum-exp, by the first lane of another warp while warp 0 selects: shift the
+  //      warps' sums to a common reference (exact powers of two times sums that carry 2^-22
+  //      already) and add them in fp64
+  if (tid == (kWarps > 1 ? kWarp : 0)) {
+    float Ref = -INFINITY;
+    for (int w = 0; w < kWarps; ++w)
+      if (sm.warp_sum[w] != 0.f) Ref = fmaxf(Ref, sm.warp_ref[w]);
+    double S = 0.0;
+    for (int w = 0; w < kWarps; ++w)
+      if (sm.warp_sum[w] != 0.f)
+        S += static_cast<double>(sm.warp_sum[w]) *
+             static_cast<double>(exp2f(sm.warp_ref[w] - Ref));
+    if constexpr (SPLIT) {
+      part->ref = Ref;
+      part->sum = S;
+    } else {
+      const double lse = lse_from_sum(Ref, S);
+      if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
+      a.out_lse[gid] = lse;
     }
-    if (lane < n && rank == k - 1) sm.tau = from_orderable(key);
-    if (lane == 0) sm.n_cand = 0;
   }
-  __syncthreads();
-  const float tau = sm.tau;
 
-  // ---- candidates: every element >= tau
-  {
-    const bool one_batch = b1 >= tau && !(b2 >= tau);
-    if (one_batch) {  // all of the thread's candidates are in its best batch
-      uint4 v[kUnroll];
-      load_checked(v, i1);
+  // ---- one warp selects (the instructions of this part are paid per warp that runs it, and a
+  //      row's candidates are a dozen elements): tau = the k-th largest thread maximum -- k
+  //      distinct elements reach it, so the row's top-k are among the elements >= tau and only
+  //      threads whose maximum reaches it can hold any.  A thread with one batch reaching tau
+  //      has that batch fetched again, a lane per vector (L2 or DRAM, one round trip for all of
+  //      them); with two or more its whole share of the row is scanned.
+  if (warp == 0) {
+    constexpr int kPerLane = kThreads / kWarp;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    if (lane == 0) sm.n_cand = 0;
+    uint32_t key[kPerLane];
 #pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int i = tid + i1 * kBatchVecs + u * kThreads;
-        if (i < nvec) push_candidates<T>(sm, v[u], vec0 + i, tau);
+    for (int q = 0; q < kPerLane; ++q) key[q] = orderable(sm.tb1[lane + 32 * q]);
+    uint32_t tau_key = kKeyNegInf;
+    for (int round = 0; round < k; ++round) {  // pop the largest remaining maximum k times
+      uint32_t m = key[0];
+#pragma unroll
+      for (int q = 1; q < kPerLane; ++q) m = max(m, key[q]);
+      tau_key = __reduce_max_sync(kFull, m);
+      const unsigned holders = __ballot_sync(kFull, m == tau_key);
+      if (lane == __ffs(holders) - 1) {
+        bool done = false;
+#pragma unroll
+        for (int q = 0; q < kPerLane; ++q)
+          if (!done && key[q] == tau_key) {
+            key[q] = 0u;  // below every key, -inf included
+            done = true;
+          }
       }
     }
-    unsigned todo = __ballot_sync(kFull, b2 >= tau);  // several batches: rescan the thread
-    while (todo) {
-      const int src = __ffs(todo) - 1;
-      todo &= todo - 1;
-      for (int i = warp * 32 + src + lane * kThreads; i < nvec; i += 32 * kThreads)
-        push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(i) * 16), vec0 + i, tau);
+    const float tau = from_orderable(tau_key < kKeyNegInf ? kKeyNegInf : tau_key);
+    int n_one = 0;
+    unsigned many[kPerLane];
+#pragma unroll
+    for (int q = 0; q < kPerLane; ++q) {
+      const int t = lane + 32 * q;
+      const bool two = sm.tb2[t] >= tau;
+      const bool one = sm.tb1[t] >= tau && !two;
+      const unsigned m1 = __ballot_sync(kFull, one);
+      if (one) sm.work[n_one + __popc(m1 & lt_mask)] = static_cast<unsigned short>(t);
+      n_one += __popc(m1);
+      many[q] = __ballot_sync(kFull, two);
+    }
+    __syncwarp();
+    for (int base = 0; base < n_one * kUnroll; base += 2 * kWarp) {  // two loads in flight
+      uint4 v[2];
+      int idx[2];
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        const int item = base + j * kWarp + lane;
+        idx[j] = -1;
+        if (item < n_one * kUnroll) {
+          const int t = sm.work[item / kUnroll];
+          const int i = t + sm.ti1[t] * kBatchVecs + (item % kUnroll) * kThreads;
+          if (i < nvec) {
+            idx[j] = i;
+            v[j] = ld_stream16(row + static_cast<size_t>(i) * 16);
+          }
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < 2; ++j)
+        if (idx[j] >= 0) push_candidates<T>(sm, v[j], vec0 + idx[j], tau);
+    }
+#pragma unroll
+    for (int q = 0; q < kPerLane; ++q) {
+      unsigned todo = many[q];
+      while (todo) {
+        const int t = __ffs(todo) - 1 + 32 * q;
+        todo &= todo - 1;
+        for (int i = t + lane * kThreads; i < nvec; i += kWarp * kThreads)
+          push_candidates<T>(sm, ld_stream16(row + static_cast<size_t>(i) * 16), vec0 + i, tau);
+      }
     }
   }
   __syncthreads();
@@ -328,26 +390,6 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
     }
   }
 
-  // ---- row log-sum-exp: shift the warps' sums to a common reference (exact powers of two
-  //      times sums that carry 2^-22 already) and add them in fp64
-  if (tid == 0) {
-    float Ref = -INFINITY;
-    for (int w = 0; w < kWarps; ++w)
-      if (sm.warp_sum[w] != 0.f) Ref = fmaxf(Ref, sm.warp_ref[w]);
-    double S = 0.0;
-    for (int w = 0; w < kWarps; ++w)
-      if (sm.warp_sum[w] != 0.f)
-        S += static_cast<double>(sm.warp_sum[w]) *
-             static_cast<double>(exp2f(sm.warp_ref[w] - Ref));
-    if constexpr (SPLIT) {
-      part->ref = Ref;
-      part->sum = S;
-    } else {
-      const double lse = lse_from_sum(Ref, S);
-      if (!isfinite(lse)) atomicOr(a.status, kStatusNonFinite);
-      a.out_lse[gid] = lse;
-    }
-  }
 }
 
 // The first CTA of a cluster merges the slices of a split row: partial sums are shifted to
