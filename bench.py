@@ -59,9 +59,9 @@ NCU_TRAFFIC = {
     # kernel: (source file, sha256 of that file at capture time, bytes per row, V of the capture)
     # from the ncu capture summarised under profiles/ (row pass, workload 2 shapes at B = 64)
     "draft_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                   "9b80b0d584d978fb10de3ec7706c5b4e528dccfda59000aa34ca2ccb52ccf1a2", (510916864 + 4050432) / 7808, 32000),
+                   "272a17195545c016c58e330703e6b63cd065fab4b0770499368178d7f1c7fbf3", (510010112 + 5054720) / 7808, 32000),
     "target_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                    "9b80b0d584d978fb10de3ec7706c5b4e528dccfda59000aa34ca2ccb52ccf1a2", (429946368 + 3444480) / 1673, 128256),
+                    "272a17195545c016c58e330703e6b63cd065fab4b0770499368178d7f1c7fbf3", (429973248 + 3899904) / 1673, 128256),
 }
 
 
