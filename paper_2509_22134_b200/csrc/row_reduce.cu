@@ -271,20 +271,45 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
 #pragma unroll
     for (int q = 0; q < kPerLane; ++q) key[q] = orderable(sm.tb1[lane + 32 * q]);
     uint32_t tau_key = kKeyNegInf;
-    for (int round = 0; round < k; ++round) {  // pop the largest remaining maximum k times
-      uint32_t m = key[0];
+    if constexpr (kPerLane == 4) {
+      // each lane sorts its four keys once; a round then takes the largest head and pops it
+      // from the first lane that holds it
+      auto order = [](uint32_t& x, uint32_t& y) {
+        const uint32_t hi = max(x, y), lo = min(x, y);
+        x = hi;
+        y = lo;
+      };
+      order(key[0], key[1]);
+      order(key[2], key[3]);
+      order(key[0], key[2]);
+      order(key[1], key[3]);
+      order(key[1], key[2]);
+      for (int round = 0; round < k; ++round) {
+        tau_key = __reduce_max_sync(kFull, key[0]);
+        const unsigned holders = __ballot_sync(kFull, key[0] == tau_key);
+        if (lane == __ffs(holders) - 1) {
+          key[0] = key[1];
+          key[1] = key[2];
+          key[2] = key[3];
+          key[3] = 0u;  // below every key, -inf included
+        }
+      }
+    } else {
+      for (int round = 0; round < k; ++round) {  // pop the largest remaining maximum k times
+        uint32_t m = key[0];
 #pragma unroll
-      for (int q = 1; q < kPerLane; ++q) m = max(m, key[q]);
-      tau_key = __reduce_max_sync(kFull, m);
-      const unsigned holders = __ballot_sync(kFull, m == tau_key);
-      if (lane == __ffs(holders) - 1) {
-        bool done = false;
+        for (int q = 1; q < kPerLane; ++q) m = max(m, key[q]);
+        tau_key = __reduce_max_sync(kFull, m);
+        const unsigned holders = __ballot_sync(kFull, m == tau_key);
+        if (lane == __ffs(holders) - 1) {
+          bool done = false;
 #pragma unroll
-        for (int q = 0; q < kPerLane; ++q)
-          if (!done && key[q] == tau_key) {
-            key[q] = 0u;  // below every key, -inf included
-            done = true;
-          }
+          for (int q = 0; q < kPerLane; ++q)
+            if (!done && key[q] == tau_key) {
+              key[q] = 0u;  // below every key, -inf included
+              done = true;
+            }
+        }
       }
     }
     const float tau = from_orderable(tau_key < kKeyNegInf ? kKeyNegInf : tau_key);
@@ -343,6 +368,7 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
     for (int c = tid; c < n_cand; c += kThreads) {
       const uint64_t key = sm.cand[c];
       int rank = 0;
+#pragma unroll 4
       for (int j = 0; j < n_cand; ++j) rank += sm.cand[j] > key ? 1 : 0;
       if (rank < k) {
         if constexpr (SPLIT) {
