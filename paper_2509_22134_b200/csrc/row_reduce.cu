@@ -60,8 +60,20 @@ namespace cg = cooperative_groups;
 #endif
 constexpr int kThreads = GTO_ROW_THREADS;
 constexpr int kWarps = kThreads / kWarp;
-constexpr int kUnroll = GTO_ROW_UNROLL;
-constexpr int kMinCtas = GTO_ROW_MIN_CTAS;  // resident CTAs per SM the register budget allows
+constexpr int kUnrollShort = GTO_ROW_UNROLL;  // vectors a thread loads together (a batch)
+constexpr int kMinCtas = GTO_ROW_MIN_CTAS;    // resident CTAs per SM the register budget allows
+// Long rows (the target vocabulary): six vectors per batch at 10 CTAs per SM.  Measured on
+// B200 on 256 KB rows, k = 1: 7257 / 6712 GB/s (burst / sustained) against 7194 / 6646; on
+// 64 KB rows the longer batches lose (6365 against 6660: five full batches and a ragged one).
+#ifndef GTO_ROW_UNROLL_LONG
+#define GTO_ROW_UNROLL_LONG 6
+#endif
+#ifndef GTO_ROW_MIN_CTAS_LONG
+#define GTO_ROW_MIN_CTAS_LONG 10
+#endif
+constexpr int kUnrollLong = GTO_ROW_UNROLL_LONG;
+constexpr int kMinCtasLong = GTO_ROW_MIN_CTAS_LONG;
+constexpr int kLongRowBytes = 128 * 1024;  // rows at least this long take the long-row variant
 constexpr int kCandCap = 512;  // with the rest of RowSmem: 12 CTAs stay within 132 KB per SM
 constexpr float kRebase = 8.f;  // largest exponent argument before a thread moves its reference
 
@@ -125,7 +137,7 @@ __device__ __forceinline__ double lse_from_sum(float ref, double S) {
 
 // One row, or with SPLIT the slice [v_begin, v_begin + v_count) of its 16-byte vectors, by the
 // whole CTA: row r of tree `tree`.  Results go to the outputs at index gid, with SPLIT to *part.
-template <typename T, bool SPLIT>
+template <typename T, bool SPLIT, int kUnroll>
 __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, int gid, int tree,
                                            int r, int v_begin, int v_count, RowPartial* part) {
   constexpr int E = T::kPerVec;
@@ -463,18 +475,18 @@ __device__ __forceinline__ void merge_row(const RowReduceArgs& a, cg::cluster_gr
 // the work list, which a bounded 1-D grid walks with a stride: the list's length is known
 // on the device only, and a CTA per possible entry would launch ~100 000 CTAs that exit at
 // once (measured: 0.54 ns each, 53 us per launch at the paper's shapes).
-template <typename T>
-__global__ void __launch_bounds__(kThreads, kMinCtas) row_reduce_kernel(RowReduceArgs a) {
+template <typename T, int U, int CTAS>
+__global__ void __launch_bounds__(kThreads, CTAS) row_reduce_kernel(RowReduceArgs a) {
   __shared__ RowSmem sm;
   if (a.list == nullptr) {
-    reduce_row<T, false>(a, sm, blockIdx.y * a.R + blockIdx.x, blockIdx.y, blockIdx.x, 0, 0, nullptr);
+    reduce_row<T, false, U>(a, sm, blockIdx.y * a.R + blockIdx.x, blockIdx.y, blockIdx.x, 0, 0, nullptr);
     return;
   }
   const int count = *a.list_count;
   for (int li = blockIdx.x; li < count; li += gridDim.x) {
     const int gid = a.list[li];
     const int tree = a.pad != 0 ? gid / a.R : 0;  // a tensor without padding rows needs no split
-    reduce_row<T, false>(a, sm, gid, tree, gid - tree * a.R, 0, 0, nullptr);
+    reduce_row<T, false, U>(a, sm, gid, tree, gid - tree * a.R, 0, 0, nullptr);
     __syncthreads();  // the row's shared state is read to the end before the next row starts
   }
 }
@@ -505,7 +517,7 @@ __global__ void __cluster_dims__(kSplit, 1, 1) __launch_bounds__(kThreads, kMinC
       tree = blockIdx.y;
       gid = tree * a.R + r;
     }
-    reduce_row<T, true>(a, sm, gid, tree, r, v_begin, v_count, &part);
+    reduce_row<T, true, kUnrollShort>(a, sm, gid, tree, r, v_begin, v_count, &part);
     cluster.sync();  // every slice's partial is complete and visible
     if (slice == 0) merge_row<T>(a, cluster, &part, gid);
     cluster.sync();  // nobody rewrites or leaves before the merge has read the partials
@@ -531,12 +543,25 @@ cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64
       row_reduce_split_kernel<F16><<<grid, block, 0, stream>>>(a);
     else
       row_reduce_split_kernel<F32><<<grid, block, 0, stream>>>(a);
-  } else if (a.dtype == GTO_BF16)
-    row_reduce_kernel<Bf16><<<grid, block, 0, stream>>>(a);
-  else if (a.dtype == GTO_F16)
-    row_reduce_kernel<F16><<<grid, block, 0, stream>>>(a);
-  else
-    row_reduce_kernel<F32><<<grid, block, 0, stream>>>(a);
+  } else {
+    const bool long_rows =
+        static_cast<size_t>(a.V) * elem_bytes(a.dtype) >= static_cast<size_t>(kLongRowBytes);
+    auto launch = [&](auto short_kernel, auto long_kernel) {
+      if (long_rows)
+        long_kernel<<<grid, block, 0, stream>>>(a);
+      else
+        short_kernel<<<grid, block, 0, stream>>>(a);
+    };
+    if (a.dtype == GTO_BF16)
+      launch(row_reduce_kernel<Bf16, kUnrollShort, kMinCtas>,
+             row_reduce_kernel<Bf16, kUnrollLong, kMinCtasLong>);
+    else if (a.dtype == GTO_F16)
+      launch(row_reduce_kernel<F16, kUnrollShort, kMinCtas>,
+             row_reduce_kernel<F16, kUnrollLong, kMinCtasLong>);
+    else
+      launch(row_reduce_kernel<F32, kUnrollShort, kMinCtas>,
+             row_reduce_kernel<F32, kUnrollLong, kMinCtasLong>);
+  }
   ++*launches;
   return cudaGetLastError();
 }
