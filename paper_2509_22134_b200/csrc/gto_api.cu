@@ -240,6 +240,7 @@ gto_status gto_build_tree(gto_ctx* ctx, const void* draft, const gto_tree* out, 
   r.out_z = ctx->top_z;
   r.status = ctx->status;
   r.split_below = split_below(ctx, r.n_rows, r.V);
+  r.sms = ctx->sms;
   {
     LaunchSpan span(ctx, GTO_K_DRAFT_ROWS, s);
     if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;
@@ -330,6 +331,7 @@ gto_status tree_reward_impl(gto_ctx* ctx, const gto_tree* tree, const void* targ
   r.out_z = nullptr;
   r.status = ctx->status;
   r.split_below = split_below(ctx, r.n_rows, r.V);
+  r.sms = ctx->sms;
   {
     LaunchSpan span(ctx, GTO_K_TARGET_ROWS, s);
     if (gto::launch_row_reduce(r, s, &ctx->launches) != cudaSuccess) return GTO_ERR_CUDA;

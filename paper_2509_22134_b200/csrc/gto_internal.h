@@ -33,6 +33,7 @@ struct RowReduceArgs {
   int32_t* status;           // device status word
   int grid_cap;              // with list: most CTAs to launch (0 = one per possible entry)
   int split_below;           // at most this many rows: split each row over a cluster (0 = never)
+  int sms;                   // multiprocessors of the device (0 = unknown)
 };
 cudaError_t launch_row_reduce(const RowReduceArgs& a, cudaStream_t stream, int64_t* launches);
 
