@@ -93,6 +93,8 @@ class DraftTree:
     row_lse: np.ndarray    # [R] draft log-sum-exp of every context row
     cut_gaps: list = field(default_factory=list)  # smallest score gap behind each layer ranking and the top-g cut
     layer_gaps: dict = field(default_factory=dict)  # depth d -> gaps between ranks (r, r+1), r < k, of layer d's ranking
+    cand_score: np.ndarray = None   # [P] score of every candidate of the pool, selected or not
+    cand_parent: np.ndarray = None  # [P] pool index of every candidate's parent, -1 = child of the root
 
 
 def context_row(d, j, k):
@@ -202,7 +204,9 @@ def build_tree(draft, D, k, g):
     return DraftTree(D=D, k=k, g=g, token=token, parent=parent, depth=depth, ctx_row=ctx,
                      slot=slot, pool=np.array(selected, dtype=np.int64), logp=logp,
                      score=score, mask=mask, row_lse=row_lse, cut_gaps=cut_gaps,
-                     layer_gaps=layer_gaps)
+                     layer_gaps=layer_gaps,
+                     cand_score=np.array([c["score"] for c in pool], dtype=np.float64),
+                     cand_parent=np.array([c["parent_pool"] for c in pool], dtype=np.int64))
 
 
 # ------------------------------------------------------------------------ O5-O6

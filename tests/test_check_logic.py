@@ -83,6 +83,44 @@ def test_a_flipped_top_g_cut_is_named_with_its_own_gap():
     assert why == [("top-g cut", pytest.approx(gap, rel=1e-12))]
 
 
+def test_the_cut_gap_is_taken_between_the_candidates_that_were_exchanged():
+    """The oracle's neighbour across the cut is a sibling with the same logit (decided by the
+    index everywhere, gap inf); the other side kept the next candidate instead, which scores
+    just below: the decision that differs is that one, with its own finite gap."""
+    for seed in range(2000):
+        rng = np.random.default_rng(seed)
+        draft = np.round(rng.normal(size=(D, K, V)) * 2.0 * 4) / 4       # a coarse grid: equal logits occur
+        tr = orc.build_tree(draft, D, K, G_NODES)
+        if tr.cut_gaps[-1] != np.inf:
+            continue
+        ranked = sorted(range(len(tr.cand_score)), key=lambda p: (-tr.cand_score[p], p))
+        x, x2, y = ranked[G_NODES - 1], ranked[G_NODES], ranked[G_NODES + 1]
+        if tr.cand_parent[x] != tr.cand_parent[x2] or tr.cand_score[x] != tr.cand_score[x2]:
+            continue
+        gap = tr.cand_score[x] - tr.cand_score[y]
+        up, related = int(tr.cand_parent[y]), False
+        while up >= 0:
+            related |= up in (x, x2)
+            up = int(tr.cand_parent[up])
+        if related or tr.cand_parent[y] == tr.cand_parent[x] or not (1e-3 < gap < 0.3):
+            continue
+        # raise the logit behind y just enough for it to pass x (and x's twin)
+        bigger = orc.build_tree(draft, D, K, G_NODES + 2)
+        at = [n for n in range(bigger.g) if int(bigger.pool[n]) == y]
+        if len(at) != 1:
+            continue
+        site = candidate_site(draft, bigger, at[0])
+        bumped = draft.copy()
+        bumped[site] += gap * 1.2 / (1.0 - np.exp(bigger.logp[at[0]]))
+        other = orc.build_tree(bumped, D, K, G_NODES)
+        if set(int(p) for p in other.pool) != (set(int(p) for p in tr.pool) - {x}) | {y}:
+            continue
+        why = ocheck.differing_decisions(tr, lists(other))
+        assert why and why[0][0] == "top-g cut" and why[0][1] == pytest.approx(gap, rel=1e-12)
+        return
+    raise AssertionError("no case found")
+
+
 def test_identical_trees_and_plain_errors():
     rng = np.random.default_rng(7)
     tr = orc.build_tree(rng.normal(size=(D, K, V)) * 2.0, D, K, G_NODES)
