@@ -62,7 +62,8 @@ def differing_decisions(tr, got):
     only the other side kept (the candidates that were actually exchanged: the oracle's own
     neighbour across the cut can be a sibling with the same logit, which nobody confuses);
     a node selected on both sides with another frontier slot is that layer's ranking, and
-    the gap reported is the largest one between the ranks the disagreement spans.
+    the gap reported is the largest one any moved candidate crossed (between its rank on
+    the two sides; two separate exchanges in one layer do not span what lies between them).
     Returns a list of (decision name, gap); empty if no ranking decision explains the
     difference (then it is a plain error)."""
     k = tr.k
@@ -83,9 +84,11 @@ def differing_decisions(tr, got):
             if d not in tr.layer_gaps:
                 return []
             rank = lambda s_: k if s_ < 0 else s_
-            ranks = [rank(mine[p][0]) for p in moved] + [rank(theirs[p][0]) for p in moved]
-            gaps = tr.layer_gaps[d][min(ranks):max(ranks)]
-            out.append((f"frontier ranking of depth {d}", float(max(gaps, default=np.inf))))
+            worst = 0.0
+            for p in moved:        # a candidate crossed every rank between its two places
+                lo, hi = sorted((rank(mine[p][0]), rank(theirs[p][0])))
+                worst = max(worst, float(max(tr.layer_gaps[d][lo:hi], default=np.inf)))
+            out.append((f"frontier ranking of depth {d}", worst))
         break
     return out
 

@@ -121,6 +121,28 @@ def test_the_cut_gap_is_taken_between_the_candidates_that_were_exchanged():
     raise AssertionError("no case found")
 
 
+def test_two_separate_exchanges_in_one_layer_do_not_span_the_ranks_between_them():
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        tr = orc.build_tree(rng.normal(size=(D, K, V)) * 2.0, D, K, G_NODES)
+        d = 2
+        at = {int(tr.slot[n]): n for n in range(tr.g) if tr.depth[n] == d and tr.slot[n] >= 0}
+        if len(at) == K:
+            break
+    # hand-made gaps between the ranks (0,1), (1,2), (2,3) of the layer: tiny, large, tiny
+    other = lists(tr)
+    other["slot"] = tr.slot.copy()
+    other["slot"][at[0]], other["slot"][at[1]] = 1, 0
+    saved = tr.layer_gaps[d]
+    tr.layer_gaps[d] = [1e-9, 5.0, 2e-9][:len(saved)] + list(saved[3:])
+    why = ocheck.differing_decisions(tr, other)
+    assert why == [(f"frontier ranking of depth {d}", 1e-9)]
+    # a candidate that moved from rank 0 to rank 2 did cross the large gap
+    other["slot"][at[0]], other["slot"][at[1]], other["slot"][at[2]] = 2, 0, 1
+    why = ocheck.differing_decisions(tr, other)
+    assert why == [(f"frontier ranking of depth {d}", 5.0)]
+
+
 def test_identical_trees_and_plain_errors():
     rng = np.random.default_rng(7)
     tr = orc.build_tree(rng.normal(size=(D, K, V)) * 2.0, D, K, G_NODES)

@@ -60,6 +60,17 @@ def test_near_tie_at_the_cut_beside_equal_siblings(harness):
     print(rep)
 
 
+def test_two_near_ties_in_one_layer(harness):
+    """Depth 4 of one tree holds two pairs of candidates 5e-12 and 3e-10 apart, with gaps of
+    several units between the pairs: each exchange is excused by its own gap."""
+    w = synth.Workload("t", B=1, V_draft=10368, V_target=10368, D=8, k=9, g=53, m=1, dtype="bf16",
+                       seed=40276, sigma_t=6.0, student_t=True)
+    p, data = harness.run_pass(w, DEV)
+    rep = harness.check_against_oracle(w, p, data, groups=[0])
+    assert rep["near_tie_trees"] >= 1
+    print(rep)
+
+
 def test_heavy_tailed_fp32_logits(harness):
     """Student-t logits at a large scale in fp32: edge log-probabilities of several hundred, where
     the fp32 outputs' own rounding is larger than the absolute tolerances."""
