@@ -89,10 +89,12 @@ def test_reduced_draft_vocabulary(harness, flags):
     print(rep)
 
 
-@pytest.mark.parametrize("case", range(16))
+@pytest.mark.parametrize("case", range(48))
 def test_random_shapes(harness, case):
     """Seeded random shapes inside the compiled limits: vocabulary (ragged tails, fewer vectors
-    than threads), depth, top-k, node budget, group size, logit type, id map, row split."""
+    than threads), depth, top-k, node budget, group size, logit type, id map, row split; from
+    case 16 on also the scale of the logits (0.3: many equal bf16 values; 6: edge
+    log-probabilities of hundreds) and heavy tails."""
     from paper_2509_22134_b200 import binding as gto
     rng = np.random.default_rng(1000 + case)
     dtype = ["bf16", "f16", "f32"][int(rng.integers(3))]
@@ -106,8 +108,11 @@ def test_random_shapes(harness, case):
     Vt = Vd + per_vec * int(rng.integers(1, 600)) if reduced else Vd
     m = int([1, 2, 4, 8][int(rng.integers(4))])
     B = m * int(rng.integers(1, 4))
+    extra = {}
+    if case >= 16:
+        extra = dict(sigma_t=float([2.5, 0.3, 6.0][int(rng.integers(3))]), student_t=bool(rng.integers(2)))
     w = synth.Workload("rnd", B=B, V_draft=Vd, V_target=Vt, D=D, k=k, g=g, m=m, dtype=dtype,
-                       seed=5000 + case)
+                       seed=5000 + case, **extra)
     flags = gto.GTO_FLAG_FORCE_ROW_SPLIT if rng.integers(2) else 0
     p, data = harness.run_pass(w, DEV, flags=flags)
     rep = harness.check_against_oracle(w, p, data, groups=list(range(B // m)))
