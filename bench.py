@@ -89,6 +89,7 @@ class ClockSampler:
     def __init__(self, device_index: int, period_s: float = 0.01):
         self.period = period_s
         self.samples, self.stamps, self.reasons, self.max_mhz = [], [], set(), None
+        self.mem_samples, self.power_samples = [], []
         self._stop = threading.Event()
         self._thread = None
         self._h = None
@@ -114,6 +115,8 @@ class ClockSampler:
                 for bit, name in self._REASONS.items():
                     if mask & bit:
                         self.reasons.add(name)
+                self.mem_samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_MEM)))
+                self.power_samples.append(int(nv.nvmlDeviceGetPowerUsage(self._h)) / 1000.0)
             except Exception:
                 pass
             self._stop.wait(self.period)
@@ -132,7 +135,9 @@ class ClockSampler:
     def summary(self):
         return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples),
+                "mem_mhz": statistics.median(self.mem_samples) if self.mem_samples else None,
+                "power_w": statistics.median(self.power_samples) if self.power_samples else None}
 
 
 # ------------------------------------------------------------------------ oracle legs
@@ -520,7 +525,8 @@ def run_gpu(args, w, rank, world, local_rank):
                              "value": world * w.B / sus_s, "gbs": step_bytes / sus_s / 1e9,
                              "frac_of_measured": step_bytes / sus_s / 1e9 / peak,
                              "frac_of_8000_nominal": step_bytes / sus_s / 1e9 / 8000.0,
-                             "sm_mhz_median": cs["sm_mhz"], "reasons": cs["reasons"],
+                             "sm_mhz_median": cs["sm_mhz"], "mem_mhz_median": cs["mem_mhz"],
+                             "power_w_median": cs["power_w"], "reasons": cs["reasons"],
                              "by_clock": by_clock(sus_steps, sus_span, sus_clocks, step_bytes)}
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"], line["parity"] = cpu_baseline_and_parity(w, data, p, b0)
