@@ -59,9 +59,9 @@ NCU_TRAFFIC = {
     # kernel: (source file, sha256 of that file at capture time, bytes per row, V of the capture)
     # from the ncu capture summarised under profiles/ (row pass, workload 2 shapes at B = 64)
     "draft_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                   "624fe344834d1626ceb33a6eb010d10e2075ecd38e525144564708108b37e7c9", (509190144 + 3539968) / 7808, 32000),
+                   "7699dc77e539aabff69340f559f8f2480559800639a44f0c23bb4d98cb358797", (509028864 + 3841536) / 7808, 32000),
     "target_rows": ("paper_2509_22134_b200/csrc/row_reduce.cu",
-                    "624fe344834d1626ceb33a6eb010d10e2075ecd38e525144564708108b37e7c9", (429943040 + 3425792) / 1673, 128256),
+                    "7699dc77e539aabff69340f559f8f2480559800639a44f0c23bb4d98cb358797", (429928448 + 3473408) / 1673, 128256),
 }
 
 

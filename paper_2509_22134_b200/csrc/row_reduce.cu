@@ -180,11 +180,13 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
     return T::max_value(acc);
   };
   auto add_terms = [&](const uint4(&v)[kUnroll]) {
+    // pairwise sum of a vector's terms, the vectors of the batch added together, then one add
+    // into the running sum: the long chain of roundings has one link per batch, not per vector
+    float batch = 0.f;
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       float f[E];
       T::unpack(v[u], f);
-      // pairwise sum of the vector's terms, then one add into the running sum
 #pragma unroll
       for (int e = 0; e < E; ++e) f[e] = ex2_approx(fmaf(f[e], kLog2e, -ref));
 #pragma unroll
@@ -192,8 +194,9 @@ __device__ __forceinline__ void reduce_row(const RowReduceArgs& a, RowSmem& sm, 
 #pragma unroll
         for (int e = 0; e < E; e += 2 * w) f[e] += f[e + w];
       }
-      s += f[0];
+      batch = u == 0 ? f[0] : batch + f[0];
     }
+    s += batch;
   };
   auto track = [&](float bm, int b) {
     const float t = bm * kLog2e;
